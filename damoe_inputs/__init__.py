@@ -1,0 +1,230 @@
+"""Seeded synthetic inputs for the distribution-aware fused-MoE path.
+
+This module only *makes inputs*: tensors of weights and activations, Dirichlet
+routing probabilities, top-k routings and gate weights.  It holds none of the
+method's arithmetic (no histogram, no Effective Experts, no expert FFN) and is
+the one piece of code that both the CPU oracle's tests and the CUDA path's
+tests/benchmarks import, so that both sides see bit-identical inputs.
+
+Two families of generators live here.
+
+* Large tensors (x, W13, W2) come from a counter-based generator written with
+  integer torch ops only, so the same call gives bit-identical bf16 values on
+  the CPU and on a CUDA device, and any expert's weights can be regenerated on
+  the host without ever holding the whole 20-30 GB weight set there.  Element
+  ``i`` of tensor ``(seed, tensor_id)`` is ``table[h16(seed, tensor_id, i)]``
+  where ``h16`` is a 16-bit field of a splitmix64-style hash and ``table`` is a
+  65 536-entry normal quantile table rounded to bf16.  This is a normal
+  distribution discretised to 2^16 quantiles (tails clipped near 4.3 sigma),
+  indistinguishable from N(0, sigma) once rounded to bf16.
+
+* Small routing inputs (Dirichlet probabilities, Gumbel-top-k expert choices,
+  softmax gate weights) are drawn on the host in fp64 with numpy's Philox
+  generator keyed by the seed, following the paper's symmetric Dirichlet routing
+  model (Section II-D, Eq. 1) with k distinct experts per token drawn without
+  replacement in proportion to p.
+"""
+from __future__ import annotations
+
+import functools
+import math
+
+import numpy as np
+import torch
+
+# tensor ids inside one seed
+TID_X, TID_W13, TID_W2 = 1, 2, 3
+
+_M1 = -0x40A7B892E31B1A47  # 0xBF58476D1CE4E5B9 as int64
+_M2 = -0x6B2FB644ECCEEE15  # 0x94D049BB133111EB as int64
+_GOLD = -0x61C8864680B583EB  # 0x9E3779B97F4A7C15 as int64
+
+
+def _lsr(z: torch.Tensor, s: int) -> torch.Tensor:
+    """Logical right shift of int64 tensors."""
+    return (z >> s) & ((1 << (64 - s)) - 1)
+
+
+def _mix64(z: torch.Tensor) -> torch.Tensor:
+    z = (z ^ _lsr(z, 30)) * _M1
+    z = (z ^ _lsr(z, 27)) * _M2
+    return z ^ _lsr(z, 31)
+
+
+def _wrap64(v: int) -> int:
+    v &= (1 << 64) - 1
+    return v - (1 << 64) if v >= (1 << 63) else v
+
+
+def _stream_key(seed: int, tensor_id: int) -> int:
+    """Scalar splitmix64 of (seed, tensor_id) computed with Python ints."""
+    def mix(z):
+        z &= (1 << 64) - 1
+        z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & ((1 << 64) - 1)
+        z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & ((1 << 64) - 1)
+        return z ^ (z >> 31)
+    return _wrap64(mix(mix(seed * 0x9E3779B97F4A7C15 + 0x1234567) ^ (tensor_id * 0xD1342543DE82EF95)))
+
+
+@functools.lru_cache(maxsize=8)
+def _quantile_table_cpu(sigma: float) -> torch.Tensor:
+    """65 536 bf16 values: sigma * Phi^-1((j + 1/2) / 65536)."""
+    from scipy.special import ndtri
+    q = ndtri((np.arange(65536, dtype=np.float64) + 0.5) / 65536.0) * sigma
+    return torch.from_numpy(q.astype(np.float32)).to(torch.bfloat16)
+
+
+_table_cache: dict = {}
+
+
+def _quantile_table(sigma: float, device) -> torch.Tensor:
+    key = (float(sigma), str(device))
+    if key not in _table_cache:
+        _table_cache[key] = _quantile_table_cpu(float(sigma)).to(device)
+    return _table_cache[key]
+
+
+def normal_bf16(seed: int, tensor_id: int, start: int, count: int, sigma: float,
+                device="cpu") -> torch.Tensor:
+    """Elements [start, start+count) of the flat bf16 tensor (seed, tensor_id).
+
+    ``start`` and ``count`` must be multiples of 4 (one 64-bit hash feeds four
+    elements).  The result is identical, bit for bit, on every device.
+    """
+    assert start % 4 == 0 and count % 4 == 0
+    table = _quantile_table(sigma, device)
+    key = _stream_key(seed, tensor_id)
+    out = torch.empty(count, dtype=torch.bfloat16, device=device)
+    chunk = 1 << 24  # hashes per piece: bounds temporaries to a few hundred MB
+    n_hash = count // 4
+    for h0 in range(0, n_hash, chunk):
+        h1 = min(n_hash, h0 + chunk)
+        ctr = torch.arange(start // 4 + h0, start // 4 + h1, dtype=torch.int64, device=device)
+        h = _mix64(ctr * _GOLD + key)
+        idx = torch.stack([h & 0xFFFF, _lsr(h, 16) & 0xFFFF, _lsr(h, 32) & 0xFFFF, _lsr(h, 48)], dim=1)
+        out[4 * h0:4 * h1] = table[idx.reshape(-1)]
+    return out
+
+
+class MoEWeights:
+    """Expert weights W13 [E, 2I, H] and W2 [E, H, I], bf16, N(0, sigma).
+
+    Rows [0, I) of W13[e] are the gate projection and rows [I, 2I) the up
+    projection.  ``expert_w13(e)`` / ``expert_w2(e)`` regenerate one expert on
+    any device; ``materialize(device)`` builds the full tensors there.
+    """
+
+    def __init__(self, seed: int, E: int, H: int, I: int, sigma: float = 0.02):
+        self.seed, self.E, self.H, self.I, self.sigma = seed, E, H, I, sigma
+
+    def expert_w13(self, e: int, device="cpu") -> torch.Tensor:
+        n = 2 * self.I * self.H
+        return normal_bf16(self.seed, TID_W13, e * n, n, self.sigma, device).view(2 * self.I, self.H)
+
+    def expert_w2(self, e: int, device="cpu") -> torch.Tensor:
+        n = self.H * self.I
+        return normal_bf16(self.seed, TID_W2, e * n, n, self.sigma, device).view(self.H, self.I)
+
+    def materialize(self, device):
+        w13 = torch.empty(self.E, 2 * self.I, self.H, dtype=torch.bfloat16, device=device)
+        w2 = torch.empty(self.E, self.H, self.I, dtype=torch.bfloat16, device=device)
+        for e in range(self.E):
+            w13[e] = self.expert_w13(e, device)
+            w2[e] = self.expert_w2(e, device)
+        return w13, w2
+
+
+def activations(seed: int, T: int, H: int, device="cpu") -> torch.Tensor:
+    """x [T, H] bf16, N(0, 1)."""
+    return normal_bf16(seed, TID_X, 0, T * H, 1.0, device).view(T, H)
+
+
+# ----------------------------------------------------------------------------
+# routing inputs (host, fp64)
+# ----------------------------------------------------------------------------
+
+def _rng(seed: int, stream: int) -> np.random.Generator:
+    return np.random.Generator(np.random.Philox(key=[seed & ((1 << 64) - 1), stream]))
+
+
+def dirichlet_log_p(alpha: float, E: int, size: int, rng: np.random.Generator) -> np.ndarray:
+    """``size`` draws of log p, p ~ Dir(alpha * 1_E)  (paper Eq. 1, symmetric case).
+
+    Gamma(alpha) variates are formed in log space as log Gamma(alpha+1) +
+    log(U)/alpha so that concentrations down to 1e-6 do not underflow.
+    """
+    g = rng.standard_gamma(alpha + 1.0, size=(size, E))
+    u = rng.random(size=(size, E))
+    u = np.maximum(u, np.finfo(np.float64).tiny)
+    lg = np.log(g) + np.log(u) / alpha
+    m = lg.max(axis=1, keepdims=True)
+    lse = m + np.log(np.exp(lg - m).sum(axis=1, keepdims=True))
+    return lg - lse
+
+
+def dirichlet_p(alpha: float, E: int, size: int, rng: np.random.Generator) -> np.ndarray:
+    return np.exp(dirichlet_log_p(alpha, E, size, rng))
+
+
+def dirichlet_sampler(seed: int):
+    """Returns ``draw(alpha, E, S) -> p[S, E]`` that restarts from the same
+    seed on every call (common random numbers across calls)."""
+    def draw(alpha: float, E: int, S: int) -> np.ndarray:
+        return dirichlet_p(alpha, E, S, _rng(seed, 7))
+    return draw
+
+
+def topk_routing(log_p: np.ndarray, T: int, k: int, rng: np.random.Generator) -> np.ndarray:
+    """ids [T, k] int32: per token, k distinct experts drawn without replacement
+    in proportion to p (Gumbel-top-k on log p), stored in draw order."""
+    E = log_p.shape[0]
+    u = rng.random(size=(T, E))
+    u = np.clip(u, np.finfo(np.float64).tiny, 1.0 - 2.0 ** -53)
+    score = log_p[None, :] - np.log(-np.log(u))
+    order = np.argsort(-score, axis=1, kind="stable")
+    return np.ascontiguousarray(order[:, :k]).astype(np.int32)
+
+
+def gate_weights(T: int, k: int, rng: np.random.Generator) -> np.ndarray:
+    """topk_weights [T, k] fp32: softmax over k iid N(0,1) logits."""
+    z = rng.standard_normal(size=(T, k))
+    z = z - z.max(axis=1, keepdims=True)
+    w = np.exp(z)
+    w /= w.sum(axis=1, keepdims=True)
+    return w.astype(np.float32)
+
+
+def routing_batch(seed: int, T: int, k: int, E: int, alpha: float):
+    """One synthetic batch's routing: (topk_ids [T,k] int32, topk_weights [T,k]
+    fp32, p [E] fp64)."""
+    log_p = dirichlet_log_p(alpha, E, 1, _rng(seed, 1))[0]
+    ids = topk_routing(log_p, T, k, _rng(seed, 2))
+    w = gate_weights(T, k, _rng(seed, 3))
+    return ids, w, np.exp(log_p)
+
+
+def uniform_routing(seed: int, T: int, k: int, E: int):
+    """Top-k of iid random logits: uniform routing without replacement (the
+    'random inputs' a static per-bucket tuner profiles with, Section IV)."""
+    ids = topk_routing(np.zeros(E), T, k, _rng(seed, 2))
+    w = gate_weights(T, k, _rng(seed, 3))
+    return ids, w
+
+
+def trace_batches(seed: int, n: int, t_max: int = 4096, a_lo: float = 0.05, a_hi: float = 10.0):
+    """Serving-trace stand-in: n (T, alpha) pairs, T log-uniform in [1, t_max],
+    alpha log-uniform in [a_lo, a_hi]."""
+    rng = _rng(seed, 11)
+    out = []
+    for _ in range(n):
+        T = int(round(math.exp(rng.random() * math.log(t_max))))
+        a = a_lo * (a_hi / a_lo) ** rng.random()
+        out.append((max(1, min(t_max, T)), float(a)))
+    return out
+
+
+CONFIGS = {
+    0: dict(E=8, k=2, H=1024, I=512),
+    1: dict(E=256, k=8, H=7168, I=2048),
+    3: dict(E=384, k=8, H=7168, I=2048),
+}

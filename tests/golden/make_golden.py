@@ -1,0 +1,49 @@
+"""Writes tests/golden/config0_oracle.txt from the CPU oracle alone.
+
+Run from the repository root:  python tests/golden/make_golden.py
+The file locks the oracle's results on the tiny configuration (E=8, top-2,
+H=1024, I=512, T=64, Dirichlet alpha=1, seed 0) so that any later change to the
+oracle's arithmetic shows up as a diff.  It imports only the seeded input
+generators and the oracle.
+"""
+import hashlib
+import os
+import sys
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
+
+from helpers import bits16, config0  # noqa: E402
+from oracle import layer, route  # noqa: E402
+
+
+def main():
+    c = config0()
+    hist = route.histogram(c.ids, c.E)
+    s1, s2, eff = route.effective_experts(hist)
+    off, perm, inv = route.offsets_and_permutation(c.ids, c.E)
+    tiles = route.tile_counts(hist, [8, 16, 32, 64, 128, 256])
+    bits, out64 = layer.moe_layer_bf16(bits16(c.x()), c.w13_bits, c.w2_bits, c.ids, c.w, c.E)
+    lines = [
+        "# written by tests/golden/make_golden.py from oracle/ only",
+        "hist " + " ".join(map(str, hist.tolist())),
+        f"sum1 {s1}", f"sum2 {s2}", f"eff_exp {eff!r}",
+        "offsets " + " ".join(map(str, off.tolist())),
+        "perm_sha256 " + hashlib.sha256(perm.astype(np.int32).tobytes()).hexdigest(),
+        "inv_sha256 " + hashlib.sha256(inv.astype(np.int32).tobytes()).hexdigest(),
+        "tiles_8_16_32_64_128_256 " + " ".join(map(str, tiles.tolist())),
+        "out_bits_sha256 " + hashlib.sha256(bits.tobytes()).hexdigest(),
+        "out64_t0_first4 " + " ".join(repr(float(v)) for v in out64[0, :4]),
+        "out64_t63_last4 " + " ".join(repr(float(v)) for v in out64[63, -4:]),
+    ]
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "config0_oracle.txt")
+    with open(path, "w") as f:
+        f.write("\n".join(lines) + "\n")
+    print("\n".join(lines))
+
+
+if __name__ == "__main__":
+    main()

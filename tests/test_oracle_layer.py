@@ -1,0 +1,153 @@
+"""Pins for the fp64 expert-layer oracle: a dense per-token brute force in a
+different formulation, reduction to a plain SwiGLU MLP checked with torch's fp64
+matmul, routing independence when all experts are equal, linearity in the gate
+weights, and the FP8 path's reduction to the bf16 path."""
+import numpy as np
+import torch
+
+import damoe_inputs as di
+from oracle import codecs, layer
+from helpers import Case, bits16, config0, max_scaled_err, rel_frobenius
+
+
+def _bf16_by_bits(a: torch.Tensor) -> torch.Tensor:
+    """binary64 -> nearest-even bfloat16 value by integer arithmetic on the binary64
+    bit pattern (normal range only): a second, independent rounding routine."""
+    b = a.numpy().view(np.uint64)
+    keep = np.uint64(45)                                   # 52 - 7 mantissa bits dropped
+    lsb = (b >> keep) & np.uint64(1)
+    r = (b + ((np.uint64(1) << np.uint64(44)) - np.uint64(1)) + lsb) >> keep << keep
+    return torch.from_numpy(r.view(np.float64).copy())
+
+
+def _dense_brute_force(case, tokens):
+    """Every expert applied to every listed token, combined with a dense [T, E]
+    weight matrix that is zero off the top-k.  Decoding and matmuls by torch."""
+    E, H, I = case.E, case.H, case.I
+    x = case.x().double()
+    D = np.zeros((case.T, E))
+    for t in range(case.T):
+        for j in range(case.k):
+            if 0 <= case.ids[t, j] < E:
+                D[t, case.ids[t, j]] += float(case.w[t, j])
+    out = np.zeros((len(tokens), H))
+    for e in range(E):
+        w13 = case.weights.expert_w13(e).double()
+        w2 = case.weights.expert_w2(e).double()
+        for n, t in enumerate(tokens):
+            g = torch.mv(w13[:I], x[t])
+            u = torch.mv(w13[I:], x[t])
+            a = (g * torch.sigmoid(g) * u)
+            h = _bf16_by_bits(a)
+            out[n] += D[t, e] * torch.mv(w2, h).numpy()
+    return out
+
+
+def test_config0_against_dense_brute_force():
+    c = config0()
+    tokens = list(range(0, 64, 3))
+    bits, out64 = layer.moe_layer_bf16(bits16(c.x()), c.w13_bits, c.w2_bits, c.ids, c.w, c.E, tokens=tokens)
+    ref = _dense_brute_force(c, tokens)
+    assert np.max(np.abs(out64 - ref)) < 1e-9
+    want = _bf16_by_bits(torch.from_numpy(ref)).to(torch.bfloat16)
+    assert np.mean(bits != bits16(want)) < 1e-3      # only exact-tie noise may differ
+
+
+def test_tokens_subset_equals_full():
+    c = config0(seed=1, T=16)
+    full, _ = layer.moe_layer_bf16(bits16(c.x()), c.w13_bits, c.w2_bits, c.ids, c.w, c.E)
+    sub, _ = layer.moe_layer_bf16(bits16(c.x()), c.w13_bits, c.w2_bits, c.ids, c.w, c.E, tokens=[5, 2, 11])
+    assert np.array_equal(sub, full[[5, 2, 11]])
+
+
+def test_single_expert_is_a_dense_swiglu_mlp():
+    T, H, I = 8, 256, 128
+    W = di.MoEWeights(9, 1, H, I, sigma=0.05)
+    x = di.activations(9, T, H)
+    ids = np.zeros((T, 1), dtype=np.int32)
+    w = np.ones((T, 1), dtype=np.float32)
+    bits, out64 = layer.moe_layer_bf16(bits16(x), lambda e: bits16(W.expert_w13(e)), lambda e: bits16(W.expert_w2(e)), ids, w, 1)
+    xd, w13, w2 = x.double(), W.expert_w13(0).double(), W.expert_w2(0).double()
+    g, u = xd @ w13[:I].T, xd @ w13[I:].T
+    h = _bf16_by_bits(torch.nn.functional.silu(g) * u)
+    ref = (h @ w2.T).numpy()
+    assert np.max(np.abs(out64 - ref)) < 1e-10
+    assert np.array_equal(bits, bits16(_bf16_by_bits(torch.from_numpy(ref)).to(torch.bfloat16)))
+
+
+def test_identical_experts_make_routing_irrelevant():
+    T, E, k, H, I = 12, 4, 2, 256, 128
+    W = di.MoEWeights(3, 1, H, I, sigma=0.05)
+    w13 = lambda e: bits16(W.expert_w13(0))
+    w2 = lambda e: bits16(W.expert_w2(0))
+    x = bits16(di.activations(3, T, H))
+    ids_a, wt, _ = di.routing_batch(1, T, k, E, 1.0)
+    ids_b, _, _ = di.routing_batch(2, T, k, E, 1.0)
+    _, a64 = layer.moe_layer_bf16(x, w13, w2, ids_a, wt, E)
+    _, b64 = layer.moe_layer_bf16(x, w13, w2, ids_b, wt, E)
+    np.testing.assert_allclose(a64, b64, rtol=0, atol=1e-12)
+    _, dense = layer.moe_layer_bf16(x, w13, w2, np.zeros((T, 1), np.int32), np.ones((T, 1), np.float32), 1)
+    np.testing.assert_allclose(a64, dense, rtol=0, atol=1e-6)   # gate weights sum to 1 in fp32 only
+
+
+def test_linear_in_gate_weights_and_slot_order():
+    c = config0(seed=2, T=8)
+    x = bits16(c.x())
+    _, base = layer.moe_layer_bf16(x, c.w13_bits, c.w2_bits, c.ids, c.w, c.E)
+    _, twice = layer.moe_layer_bf16(x, c.w13_bits, c.w2_bits, c.ids, (2 * c.w).astype(np.float32), c.E)
+    np.testing.assert_allclose(twice, 2 * base, rtol=1e-14)
+    zb, z64 = layer.moe_layer_bf16(x, c.w13_bits, c.w2_bits, c.ids, np.zeros_like(c.w), c.E)
+    assert np.all(z64 == 0) and np.all(zb == 0)
+    _, swapped = layer.moe_layer_bf16(x, c.w13_bits, c.w2_bits, c.ids[:, ::-1], c.w[:, ::-1], c.E)
+    np.testing.assert_allclose(swapped, base, rtol=1e-12, atol=1e-14)
+
+
+def test_invalid_id_contributes_nothing():
+    c = config0(seed=4, T=4)
+    x = bits16(c.x())
+    ids = c.ids.copy()
+    ids[1, 0] = -1
+    ids[2, 1] = c.E
+    wz = c.w.copy()
+    wz[1, 0] = 0
+    wz[2, 1] = 0
+    _, a = layer.moe_layer_bf16(x, c.w13_bits, c.w2_bits, ids, c.w, c.E)
+    _, b = layer.moe_layer_bf16(x, c.w13_bits, c.w2_bits, c.ids, wz, c.E)
+    np.testing.assert_allclose(a, b, rtol=0, atol=0)
+
+
+def test_swiglu_values():
+    g = np.array([0.0, 1.0, -1.0, 30.0])
+    u = np.array([5.0, 2.0, 2.0, 1.0])
+    want = np.array([0.0, 2 / (1 + np.exp(-1.0)), -2 / (1 + np.exp(1.0)), 30.0 / (1 + np.exp(-30.0))])
+    np.testing.assert_allclose(layer.swiglu(g, u), want, rtol=1e-15)
+
+
+def test_fp8_with_unit_scales_equals_bf16_path():
+    # values exactly representable in E4M3 and small enough that h needs no rescale issue
+    rng = np.random.default_rng(0)
+    T, E, k, H, I = 6, 3, 2, 128, 128
+    codes = lambda shape: rng.integers(0, 0x30, size=shape, dtype=np.uint8) | (rng.integers(0, 2, size=shape, dtype=np.uint8) << 7)
+    xq, w13q, w2q = codes((T, H)), codes((E, 2 * I, H)), codes((E, H, I))
+    ones = lambda *s: np.ones(s, dtype=np.float32)
+    ids, w, _ = di.routing_batch(0, T, k, E, 1.0)
+    to_bf16 = lambda q: codecs.bf16_rne(codecs.e4m3_decode(q))
+    _, ref = layer.moe_layer_bf16(to_bf16(xq), to_bf16(w13q), to_bf16(w2q), ids, w, E)
+    _, got = layer.moe_layer_fp8(xq, ones(T, 1), w13q, ones(E, 2, 1), w2q, ones(E, 1, 1), ids, w, E)
+    # the fp8 path additionally re-quantises h to E4M3 (3 mantissa bits): bounded relative error
+    assert rel_frobenius(got, ref) < 0.04
+    # and with h already exactly representable (zero activations) both are exactly zero
+    _, z = layer.moe_layer_fp8(np.zeros_like(xq), ones(T, 1), w13q, ones(E, 2, 1), w2q, ones(E, 1, 1), ids, w, E)
+    assert np.all(z == 0)
+
+
+def test_quantize_act_groups():
+    h = np.zeros((2, 256))
+    h[0, :128] = np.linspace(-7, 7, 128)
+    h[1, 128:] = 448.0
+    codes, s = layer.quantize_act_e4m3(h)
+    assert s.shape == (2, 2) and s.dtype == np.float32
+    assert s[0, 0] == np.float32(7.0) / np.float32(448.0) and s[0, 1] == 1.0 and s[1, 1] == 1.0
+    assert np.all(codecs.e4m3_decode(codes[1, 128:]) == 448.0)
+    deq = codecs.e4m3_decode(codes[0, :128]) * float(s[0, 0])
+    assert np.max(np.abs(deq - h[0, :128])) <= 7 / 448 * 16 + 1e-12   # half a quantum of the top binade
