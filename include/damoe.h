@@ -1,0 +1,178 @@
+/*
+ * damoe.h - C ABI of the distribution-aware fused-MoE library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the one hot path of "Decoding the Skew: Distribution-Aware MoE
+ * Inference with Adaptive Kernel Dispatch": given the router's top-k output on the GPU, pick
+ * and launch the fused-MoE kernel variant that suits the observed routing distribution,
+ * without any CPU-GPU synchronisation (paper Section IV), and run the expert layer.
+ *
+ * Conventions that hold for every entry point
+ *   - "dev" pointers are device pointers on the context's device, "host" pointers are host
+ *     pointers.  All are owned by the caller; the library never frees or reallocates them.
+ *   - The library owns only its context: scratch workspace sized at damoe_create, the device
+ *     copy of the tuning table, and the captured dispatch graphs.
+ *   - Every call returns an int status (DAMOE_OK == 0).  Nothing throws, nothing exits.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     damoe_route_stats and damoe_fused_moe only enqueue work on it and never synchronise.
+ *   - There is no CPU fallback: an unsupported shape is an error.
+ *
+ * Tensor layouts (all row-major, innermost dimension last)
+ *   x            [T, H]      bf16          activations
+ *   w13          [E, 2I, H]  bf16          rows [0, I) of an expert = gate projection (goes
+ *                                          through SiLU), rows [I, 2I) = up projection
+ *   w2           [E, H, I]   bf16          down projection
+ *   topk_ids     [T, k]      int32         expert ids as drawn by the router; an id outside
+ *                                          [0, E) is skipped, contributes zero to `out`, and
+ *                                          sets DAMOE_STATUS_BAD_ID; duplicates are legal
+ *   topk_weights [T, k]      float32       used as given (no renormalisation)
+ *   out          [T, H]      bf16          out[t] = bf16( sum_j w[t,j] * W2[e] . bf16(silu(g) * u) )
+ */
+#ifndef DAMOE_H
+#define DAMOE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct damoe_ctx damoe_ctx;
+
+enum {
+  DAMOE_OK = 0,
+  DAMOE_ERR_INVALID_ARG = 1,       /* NULL pointer, negative size, T > max_T, bad variant id */
+  DAMOE_ERR_UNSUPPORTED_SHAPE = 2, /* H or I not a multiple of 128, E > 1024, k > 32, ... */
+  DAMOE_ERR_CUDA = 3,              /* a CUDA runtime/driver call failed; see damoe_last_error */
+  DAMOE_ERR_TABLE_FORMAT = 4,      /* tuning-table bytes are malformed */
+  DAMOE_ERR_TABLE_MISMATCH = 5,    /* table was built for another (E, k, H, I, dtype, variants) */
+  DAMOE_ERR_WORKSPACE = 6,         /* workspace allocation failed / size beyond a fixed limit */
+  DAMOE_ERR_DEVICE_STATUS = 7      /* a kernel reported a problem; see damoe_debug_fetch */
+};
+
+enum { DAMOE_BF16 = 0, DAMOE_FP8_E4M3_BLOCK128 = 1 };
+
+/* `variant` argument of damoe_fused_moe */
+#define DAMOE_VARIANT_AUTO (-1)   /* device-side selection from the loaded table (built-in cost model if none) */
+#define DAMOE_VARIANT_STATIC (-2) /* the table's static per-token-count-bucket choice: the comparison baseline */
+
+/* how DAMOE_VARIANT_AUTO reaches the chosen kernel (all three stay on the device) */
+enum {
+  DAMOE_DISPATCH_BRANCH = 0,     /* one persistent kernel per GEMM that branches on the variant id */
+  DAMOE_DISPATCH_PREDICATED = 1, /* every variant is launched; all but the chosen one exit at once */
+  DAMOE_DISPATCH_GRAPH_SWITCH = 2 /* CUDA-graph conditional SWITCH node (paper Section IV-C) */
+};
+
+/* tuning-table selection modes */
+enum { DAMOE_MODE_EXEMPLAR = 0, DAMOE_MODE_EFFEXP_BINS = 1, DAMOE_MODE_COST = 2 };
+
+/* bits of the device status word */
+#define DAMOE_STATUS_BAD_ID 1u        /* an expert id outside [0, E) was skipped */
+#define DAMOE_STATUS_NO_VALID_ID 2u   /* no valid id at all: Effective Experts reported as 0 */
+#define DAMOE_STATUS_WAIT_TIMEOUT 4u  /* a bounded barrier wait inside a GEMM kernel gave up */
+#define DAMOE_STATUS_BAD_VARIANT 8u   /* the selector produced an id outside the variant list */
+
+/*
+ * Context.  Allocates, once, all scratch the path needs for up to max_T tokens: routing
+ * metadata, the permuted activations [max_T*k, H] bf16, the intermediate h [max_T*k, I] bf16
+ * and the per-pair down-projection results [max_T*k, H] fp32.  `device` becomes the current
+ * device of the calling thread.  Requirements: 1 <= k <= 32, 1 <= E <= 1024, H and I
+ * multiples of 128.  dtype DAMOE_FP8_E4M3_BLOCK128 is declared but not implemented yet:
+ * damoe_create returns DAMOE_ERR_UNSUPPORTED_SHAPE for it.
+ */
+int damoe_create(damoe_ctx** ctx, int device, int max_T, int k, int E, int H, int I, int dtype);
+int damoe_destroy(damoe_ctx* ctx);
+
+/* Text of the last error recorded on this context (never NULL; owned by the context). */
+const char* damoe_last_error(const damoe_ctx* ctx);
+
+/*
+ * Per-expert token histogram t_i and the Effective Experts statistic
+ *     eff_exp = (sum_i t_i)^2 / sum_i t_i^2                      (paper Section III-A, Eq. 2)
+ * topk_ids: dev [T, k] int32.  hist: dev [E] int32 (written).  eff_exp: dev [1] double
+ * (written; both sums are exact integers and the one division is IEEE binary64, so the value
+ * is bit-identical to a CPU evaluation; 0 when no id is valid).  k and E must equal the
+ * context's.  T == 0 writes a zero histogram and eff_exp 0.  Enqueues on `stream`; no sync.
+ */
+int damoe_route_stats(damoe_ctx* ctx, const int32_t* topk_ids, int T, int k, int E,
+                      int32_t* hist, double* eff_exp, void* stream);
+
+/*
+ * The whole layer (paper Section IV, Fig. 9(b) steps 5-6 plus the expert computation of
+ * Section II-C): histogram and Effective Experts, stable grouping of (token, slot) pairs by
+ * expert, per-variant padded-tile counts  tiles_v = sum_e ceil(t_e / N_v),  device-side choice
+ * of the kernel variant, grouped gate/up GEMM with fused SwiGLU, grouped down GEMM with the
+ * routing weight fused into its epilogue, and the top-k unpermute-reduce in fixed slot order.
+ *
+ * x, w13, w2, topk_ids, topk_weights, out: dev, layouts above.  0 <= T <= max_T; T == 0 returns
+ * DAMOE_OK and touches nothing.  variant: an id in [0, damoe_variant_count()), or
+ * DAMOE_VARIANT_AUTO, or DAMOE_VARIANT_STATIC.  The token-count bucket is the smallest table
+ * bucket >= T, else the largest (T is a host-known shape, so this costs no synchronisation).
+ * Enqueues on `stream`; never synchronises; safe to capture in a CUDA graph unless the
+ * dispatch mode is DAMOE_DISPATCH_GRAPH_SWITCH (which launches an internal graph).
+ * Calls on one context must not overlap on the GPU: they share the context's workspace.
+ */
+int damoe_fused_moe(damoe_ctx* ctx, const void* x, const void* w13, const void* w2,
+                    const int32_t* topk_ids, const float* topk_weights, int T, int variant,
+                    void* out, void* stream);
+
+/*
+ * End-to-end form with the per-step tensors on the HOST: x_host [T,H] bf16, topk_ids_host
+ * [T,k] int32, topk_weights_host [T,k] float32 are copied to the device, the layer runs, and
+ * out_host [T,H] bf16 is copied back; the call returns after the result has arrived
+ * (it synchronises `stream`).  Expert weights w13/w2 stay device-resident (dev pointers).
+ * Pinned host memory makes the copies asynchronous; pageable memory works but is slower.
+ */
+int damoe_fused_moe_host(damoe_ctx* ctx, const void* x_host, const void* w13, const void* w2,
+                         const int32_t* topk_ids_host, const float* topk_weights_host, int T,
+                         int variant, void* out_host, void* stream);
+
+/* FP8 block scales (dtype == DAMOE_FP8_E4M3_BLOCK128 only): x_scale dev [T, H/128],
+ * w13_scale dev [E, 2I/128, H/128], w2_scale dev [E, H/128, I/128], all float32.
+ * Not implemented yet: returns DAMOE_ERR_UNSUPPORTED_SHAPE. */
+int damoe_set_fp8_scales(damoe_ctx* ctx, const float* x_scale, const float* w13_scale,
+                         const float* w2_scale);
+
+/*
+ * Offline tuning table (paper Section IV-A): per token-count bucket, the exemplars (sorted,
+ * L2-normalised per-expert count vectors, stored as round(e_i * 2^30)) paired with the id of
+ * the fastest kernel, plus the static per-bucket choice of the baseline.  `bytes` is a host
+ * buffer in the format written by the Python module paper_2607_23099_b200.tuning (little
+ * endian; header "DAMOETB1").  The bytes are parsed, checked against the context's
+ * (E, k, H, I, dtype) and the library's variant count, copied, and uploaded once.  Loading a
+ * new table replaces the old one.  This call synchronises the device.
+ */
+int damoe_load_tuning_table(damoe_ctx* ctx, const void* bytes, size_t nbytes);
+
+/* Select how DAMOE_VARIANT_AUTO dispatches (default DAMOE_DISPATCH_BRANCH). */
+int damoe_set_dispatch(damoe_ctx* ctx, int dispatch_mode);
+
+/* The kernel family.  tile_n = token-tile width N_v (the paper's Tile-N), tile_m = weight rows
+ * per MMA tile, cta_group = 1 or 2 CTAs per tile, stages = shared-memory pipeline depth of
+ * the gate/up GEMM.  Any out-pointer may be NULL. */
+int damoe_variant_count(void);
+int damoe_variant_info(int id, int* tile_n, int* tile_m, int* cta_group, int* stages);
+
+/*
+ * Test / diagnostic only - synchronises the device.  Copies the routing metadata of the last
+ * damoe_fused_moe call to host buffers (any pointer may be NULL): offsets [E+1], perm [T*k]
+ * (sorted position -> flat pair index t*k+j; positions past the valid count hold -1),
+ * inv [T*k] (-1 for skipped pairs), tiles [damoe_variant_count()], the chosen variant id,
+ * and the status bits (cleared by the read).
+ */
+int damoe_debug_fetch(damoe_ctx* ctx, int32_t* offsets, int32_t* perm, int32_t* inv,
+                      int32_t* tiles, int32_t* variant_id, uint32_t* status_bits);
+
+/*
+ * Dispatch microbenchmark (paper Section V-C, Table III): a producer kernel computes a value
+ * that selects one of two trivial follow-up kernels.  Times `iters` repetitions of each of
+ * three paths and writes the mean microseconds per repetition: us[0] copy the value to the
+ * host and branch on the CPU, us[1] CUDA-graph conditional SWITCH on the GPU, us[2] a fixed
+ * graph with no branch.  Synchronises.  us: host [3].
+ */
+int damoe_dispatch_microbench(int device, int iters, float* us);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DAMOE_H */

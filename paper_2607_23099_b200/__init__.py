@@ -1,0 +1,171 @@
+"""Python binding of libdamoe (include/damoe.h): argument marshalling only.
+
+Every step of the path - histogram, Effective Experts, permutation, variant selection, both
+grouped GEMMs and the unpermute-reduce - runs in the library's CUDA kernels.  PyTorch is used
+for device memory and streams.  There is no CPU fallback: if the shared library is missing or
+does not load, importing this package raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdamoe.so")
+
+OK = 0
+BF16, FP8_E4M3_BLOCK128 = 0, 1
+VARIANT_AUTO, VARIANT_STATIC = -1, -2
+DISPATCH_BRANCH, DISPATCH_PREDICATED, DISPATCH_GRAPH_SWITCH = 0, 1, 2
+MODE_EXEMPLAR, MODE_EFFEXP_BINS, MODE_COST = 0, 1, 2
+STATUS_BAD_ID, STATUS_NO_VALID_ID, STATUS_WAIT_TIMEOUT, STATUS_BAD_VARIANT = 1, 2, 4, 8
+
+EXPORTS = [
+    "damoe_create", "damoe_destroy", "damoe_last_error", "damoe_route_stats", "damoe_fused_moe",
+    "damoe_fused_moe_host", "damoe_set_fp8_scales", "damoe_load_tuning_table", "damoe_set_dispatch",
+    "damoe_variant_count", "damoe_variant_info", "damoe_debug_fetch", "damoe_dispatch_microbench",
+]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2607_23099_b200.build` "
+            "(needs nvcc with sm_100a support); there is no fallback path")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, cp = ctypes.c_void_p, ctypes.c_int, ctypes.c_char_p
+    lib.damoe_create.argtypes = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, i32, i32]
+    lib.damoe_destroy.argtypes = [vp]
+    lib.damoe_last_error.argtypes = [vp]
+    lib.damoe_last_error.restype = cp
+    lib.damoe_route_stats.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
+    lib.damoe_fused_moe.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
+    lib.damoe_fused_moe_host.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
+    lib.damoe_set_fp8_scales.argtypes = [vp, vp, vp, vp]
+    lib.damoe_load_tuning_table.argtypes = [vp, ctypes.c_char_p, ctypes.c_size_t]
+    lib.damoe_set_dispatch.argtypes = [vp, i32]
+    lib.damoe_variant_count.argtypes = []
+    lib.damoe_variant_info.argtypes = [i32] + [ctypes.POINTER(i32)] * 4
+    lib.damoe_debug_fetch.argtypes = [vp] * 7
+    lib.damoe_dispatch_microbench.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_float)]
+    for name in EXPORTS:
+        if name != "damoe_last_error":
+            getattr(lib, name).restype = i32
+    return lib
+
+
+_lib = _load()
+
+
+class DamoeError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"damoe error {code}: {msg}")
+        self.code = code
+
+
+def variant_count() -> int:
+    return _lib.damoe_variant_count()
+
+
+def variant_info(vid: int) -> dict:
+    n, m, g, s = (ctypes.c_int() for _ in range(4))
+    rc = _lib.damoe_variant_info(vid, ctypes.byref(n), ctypes.byref(m), ctypes.byref(g), ctypes.byref(s))
+    if rc != OK:
+        raise DamoeError(rc, f"no variant {vid}")
+    return dict(id=vid, tile_n=n.value, tile_m=m.value, cta_group=g.value, stages=s.value)
+
+
+def tile_ns() -> list:
+    return [variant_info(v)["tile_n"] for v in range(variant_count())]
+
+
+def dispatch_microbench(iters: int = 200, device: int = 0) -> dict:
+    us = (ctypes.c_float * 3)()
+    rc = _lib.damoe_dispatch_microbench(device, iters, us)
+    if rc != OK:
+        raise DamoeError(rc, "dispatch microbenchmark failed")
+    return dict(host_branch_us=us[0], conditional_graph_us=us[1], fixed_graph_us=us[2])
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+class DAMoE:
+    """One context = one layer shape (k, E, H, I) with scratch for up to max_T tokens."""
+
+    def __init__(self, max_T: int, k: int, E: int, H: int, I: int, dtype: int = BF16, device: int = 0):
+        self.max_T, self.k, self.E, self.H, self.I, self.device = max_T, k, E, H, I, device
+        self._ctx = ctypes.c_void_p()
+        rc = _lib.damoe_create(ctypes.byref(self._ctx), device, max_T, k, E, H, I, dtype)
+        if rc != OK:
+            self._ctx = ctypes.c_void_p()
+            raise DamoeError(rc, "damoe_create failed")
+
+    def close(self):
+        if self._ctx:
+            _lib.damoe_destroy(self._ctx)
+            self._ctx = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int):
+        if rc != OK:
+            raise DamoeError(rc, _lib.damoe_last_error(self._ctx).decode())
+
+    def route_stats(self, topk_ids: torch.Tensor, hist=None, eff_exp=None, stream=None):
+        T = topk_ids.shape[0]
+        dev = topk_ids.device
+        hist = torch.empty(self.E, dtype=torch.int32, device=dev) if hist is None else hist
+        eff_exp = torch.empty(1, dtype=torch.float64, device=dev) if eff_exp is None else eff_exp
+        self._check(_lib.damoe_route_stats(self._ctx, _ptr(topk_ids), T, self.k, self.E, _ptr(hist), _ptr(eff_exp),
+                                           _stream_ptr(stream)))
+        return hist, eff_exp
+
+    def fused_moe(self, x, w13, w2, topk_ids, topk_weights, variant: int = VARIANT_AUTO, out=None, stream=None):
+        T = x.shape[0]
+        out = torch.empty(T, self.H, dtype=torch.bfloat16, device=x.device) if out is None else out
+        self._check(_lib.damoe_fused_moe(self._ctx, _ptr(x), _ptr(w13), _ptr(w2), _ptr(topk_ids), _ptr(topk_weights),
+                                         T, variant, _ptr(out), _stream_ptr(stream)))
+        return out
+
+    def fused_moe_host(self, x_host, w13, w2, topk_ids_host, topk_weights_host, variant: int = VARIANT_AUTO,
+                       out_host=None, stream=None):
+        T = x_host.shape[0]
+        if out_host is None:
+            out_host = torch.empty(T, self.H, dtype=torch.bfloat16).pin_memory()
+        self._check(_lib.damoe_fused_moe_host(self._ctx, _ptr(x_host), _ptr(w13), _ptr(w2), _ptr(topk_ids_host),
+                                              _ptr(topk_weights_host), T, variant, _ptr(out_host),
+                                              _stream_ptr(stream)))
+        return out_host
+
+    def load_tuning_table(self, blob: bytes):
+        self._check(_lib.damoe_load_tuning_table(self._ctx, blob, len(blob)))
+
+    def set_dispatch(self, mode: int):
+        self._check(_lib.damoe_set_dispatch(self._ctx, mode))
+
+    def debug_fetch(self, T: int) -> dict:
+        """Routing metadata of the last fused_moe call (synchronises)."""
+        P, V = T * self.k, variant_count()
+        off = torch.empty(self.E + 1, dtype=torch.int32)
+        perm = torch.empty(P, dtype=torch.int32)
+        inv = torch.empty(P, dtype=torch.int32)
+        tiles = torch.empty(V, dtype=torch.int32)
+        vid = torch.empty(1, dtype=torch.int32)
+        status = torch.empty(1, dtype=torch.int32)
+        self._check(_lib.damoe_debug_fetch(self._ctx, _ptr(off), _ptr(perm), _ptr(inv), _ptr(tiles), _ptr(vid),
+                                           _ptr(status)))
+        return dict(offsets=off.numpy(), perm=perm.numpy(), inv=inv.numpy(), tiles=tiles.numpy(),
+                    variant_id=int(vid[0]), status=int(status[0]) & 0xFFFFFFFF)

@@ -1,0 +1,487 @@
+// The C ABI (include/damoe.h): context, tuning-table loading, and the host side of the layer
+// call.  The host side only validates, picks the token-count bucket from T (a shape the host
+// knows) and enqueues kernels; every routing-dependent decision is taken on the device.
+#include <cstdarg>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace damoe;
+
+struct TableBucket {
+  int T = 0;
+  int static_variant = 0;
+  int n_ex = 0;
+  int n_bins = 0;
+  uint64_t bin_den = 1;
+  size_t off_ex = 0, off_exv = 0, off_bnum = 0, off_binv = 0, off_cost = 0;  // byte offsets into the device blob
+};
+
+struct damoe_ctx {
+  int device = 0, max_T = 0, k = 0, E = 0, H = 0, I = 0, dtype = 0;
+  int max_P = 0, sm_count = 0, dispatch = DAMOE_DISPATCH_BRANCH, last_T = 0;
+  Workspace ws{};
+  void* arena = nullptr;  // one allocation backing every workspace pointer
+  // tuning table
+  bool has_table = false;
+  int table_mode = DAMOE_MODE_COST;
+  std::vector<TableBucket> buckets;
+  uint8_t* table_blob = nullptr;
+  int64_t* default_cost = nullptr;  // [4, V] built-in cost model used when no table is loaded
+  // tensor maps: activations are fixed (workspace), weights are cached by pointer
+  CUtensorMap map_x[kNumVariants], map_h[kNumVariants];
+  CUtensorMap map_w13, map_w2;
+  const void* cached_w13 = nullptr;
+  const void* cached_w2 = nullptr;
+  // staging for the host-buffer entry point
+  void *st_x = nullptr, *st_ids = nullptr, *st_w = nullptr, *st_out = nullptr;
+  char err[256] = "";
+};
+
+namespace {
+
+int fail(damoe_ctx* c, int code, const char* fmt, ...) {
+  if (c) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(c->err, sizeof(c->err), fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+
+#define DAMOE_CUDA(c, expr)                                                                      \
+  do {                                                                                           \
+    cudaError_t e_ = (expr);                                                                     \
+    if (e_ != cudaSuccess) return fail((c), DAMOE_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
+  } while (0)
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 matrix [rows, cols] row-major, box = 64 columns (128 bytes) x box_rows, 128-byte swizzle.
+int make_map(damoe_ctx* c, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return fail(c, DAMOE_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(kBK), box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(c, DAMOE_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+  return DAMOE_OK;
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Built-in cost coefficients (picoseconds) from the roofline constants of a B200: one
+// expert's weights streamed from HBM, one extra pass served by L2, and tensor time per padded
+// token column with small tiles running the MMA pipe below peak.
+void default_cost_model(const damoe_ctx* c, int64_t* cost) {
+  const double wbytes = 3.0 * c->H * c->I * 2.0;
+  const double flops_col = 6.0 * c->H * c->I;
+  for (int v = 0; v < kNumVariants; ++v) {
+    const int n = variant_desc(v).tile_n;
+    const double eff = 0.75 * (n >= 128 ? 1.0 : n / 128.0);
+    cost[0 * kNumVariants + v] = 0;
+    cost[1 * kNumVariants + v] = static_cast<int64_t>(wbytes / 6.5e12 * 1e12);
+    cost[2 * kNumVariants + v] = static_cast<int64_t>(wbytes / 13e12 * 1e12);
+    cost[3 * kNumVariants + v] = static_cast<int64_t>(flops_col / (1.4e15 * eff) * 1e12);
+  }
+}
+
+int pick_bucket(const damoe_ctx* c, int T) {
+  int best = -1, largest = 0;
+  for (int i = 0; i < (int)c->buckets.size(); ++i) {
+    if (c->buckets[i].T >= T && (best < 0 || c->buckets[i].T < c->buckets[best].T)) best = i;
+    if (c->buckets[i].T > c->buckets[largest].T) largest = i;
+  }
+  return best >= 0 ? best : largest;
+}
+
+constexpr int kDefaultStaticVariant = 2;
+
+// Fills the selector arguments for this call; returns the host-known variant (>= 0) when the
+// choice does not depend on the routing, else -1.
+int make_selector(const damoe_ctx* c, int T, int variant, SelectorArgs* sel) {
+  memset(sel, 0, sizeof(*sel));
+  sel->forced = -1;
+  sel->mode = DAMOE_MODE_COST;
+  sel->cost = c->default_cost;
+  sel->bin_den = 1;
+  const TableBucket* b = c->has_table ? &c->buckets[pick_bucket(c, T)] : nullptr;
+  if (variant >= 0) {
+    sel->forced = variant;
+  } else if (variant == DAMOE_VARIANT_STATIC) {
+    sel->forced = b ? b->static_variant : kDefaultStaticVariant;
+  } else if (b) {
+    sel->mode = c->table_mode;
+    sel->n_exemplars = b->n_ex;
+    sel->exemplars = reinterpret_cast<const int32_t*>(c->table_blob + b->off_ex);
+    sel->ex_variant = reinterpret_cast<const int32_t*>(c->table_blob + b->off_exv);
+    sel->n_bins = b->n_bins;
+    sel->bin_num = reinterpret_cast<const uint64_t*>(c->table_blob + b->off_bnum);
+    sel->bin_den = b->bin_den;
+    sel->bin_variant = reinterpret_cast<const int32_t*>(c->table_blob + b->off_binv);
+    sel->cost = reinterpret_cast<const int64_t*>(c->table_blob + b->off_cost);
+  }
+  return sel->forced;
+}
+
+struct Reader {
+  const uint8_t* p;
+  size_t left;
+  bool ok = true;
+  template <class T>
+  T get() {
+    T v{};
+    if (left < sizeof(T)) {
+      ok = false;
+      return v;
+    }
+    memcpy(&v, p, sizeof(T));
+    p += sizeof(T);
+    left -= sizeof(T);
+    return v;
+  }
+  const uint8_t* take(size_t n) {
+    if (left < n) {
+      ok = false;
+      return nullptr;
+    }
+    const uint8_t* r = p;
+    p += n;
+    left -= n;
+    return r;
+  }
+};
+
+}  // namespace
+
+extern "C" {
+
+int damoe_variant_count(void) { return kNumVariants; }
+
+int damoe_variant_info(int id, int* tile_n, int* tile_m, int* cta_group, int* stages) {
+  if (id < 0 || id >= kNumVariants) return DAMOE_ERR_INVALID_ARG;
+  const VariantDesc d = variant_desc(id);
+  if (tile_n) *tile_n = d.tile_n;
+  if (tile_m) *tile_m = d.tile_m;
+  if (cta_group) *cta_group = d.cta_group;
+  if (stages) *stages = d.stages13;
+  return DAMOE_OK;
+}
+
+const char* damoe_last_error(const damoe_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+int damoe_create(damoe_ctx** out, int device, int max_T, int k, int E, int H, int I, int dtype) {
+  if (!out) return DAMOE_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (max_T < 1 || k < 1 || E < 1 || H < 1 || I < 1) return DAMOE_ERR_INVALID_ARG;
+  if (dtype != DAMOE_BF16) return DAMOE_ERR_UNSUPPORTED_SHAPE;
+  if (k > kMaxK || E > kMaxE || H % 128 != 0 || I % 128 != 0) return DAMOE_ERR_UNSUPPORTED_SHAPE;
+  if (static_cast<long long>(max_T) * k > 131072) return DAMOE_ERR_WORKSPACE;  // keeps the selector's integers in 64 bits
+  damoe_ctx* c = new (std::nothrow) damoe_ctx();
+  if (!c) return DAMOE_ERR_WORKSPACE;
+  c->device = device; c->max_T = max_T; c->k = k; c->E = E; c->H = H; c->I = I; c->dtype = dtype;
+  c->max_P = max_T * k;
+  auto bail = [&](int code) {
+    damoe_destroy(c);
+    return code;
+  };
+  if (cudaSetDevice(device) != cudaSuccess) return bail(DAMOE_ERR_CUDA);
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return bail(DAMOE_ERR_CUDA);
+  if (prop.major != 10) return bail(DAMOE_ERR_UNSUPPORTED_SHAPE);  // tcgen05 kernels: sm_100a only
+  c->sm_count = prop.multiProcessorCount;
+  if (gemm_configure() != cudaSuccess) return bail(DAMOE_ERR_CUDA);
+
+  // one arena; 1024-byte aligned slices
+  const size_t P = c->max_P;
+  const int nblk = (c->max_P + kPairsPerBlock - 1) / kPairsPerBlock;
+  size_t off = 0;
+  auto carve = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 1024);
+    return o;
+  };
+  const size_t o_hist = carve(sizeof(int32_t) * E), o_sums = carve(16), o_eff = carve(8),
+               o_off = carve(sizeof(int32_t) * (E + 1)), o_perm = carve(sizeof(int32_t) * P),
+               o_inv = carve(sizeof(int32_t) * P), o_ws = carve(sizeof(float) * P),
+               o_tiles = carve(sizeof(int32_t) * kNumVariants),
+               o_pref = carve(sizeof(int32_t) * kNumVariants * (E + 1)), o_act = carve(4), o_var = carve(4),
+               o_stat = carve(4), o_bh = carve(sizeof(int32_t) * nblk * E), o_cost = carve(8 * 4 * kNumVariants),
+               o_xp = carve(2 * P * H), o_h = carve(2 * P * I), o_y = carve(4 * P * H),
+               o_sx = carve(2 * static_cast<size_t>(max_T) * H), o_sid = carve(4 * P), o_sw = carve(4 * P),
+               o_so = carve(2 * static_cast<size_t>(max_T) * H);
+  if (cudaMalloc(&c->arena, off) != cudaSuccess) {
+    c->arena = nullptr;
+    return bail(DAMOE_ERR_WORKSPACE);
+  }
+  if (cudaMemset(c->arena, 0, off) != cudaSuccess) return bail(DAMOE_ERR_CUDA);
+  uint8_t* a = static_cast<uint8_t*>(c->arena);
+  c->ws.hist = reinterpret_cast<int32_t*>(a + o_hist);
+  c->ws.sums = reinterpret_cast<unsigned long long*>(a + o_sums);
+  c->ws.eff = reinterpret_cast<double*>(a + o_eff);
+  c->ws.offsets = reinterpret_cast<int32_t*>(a + o_off);
+  c->ws.perm = reinterpret_cast<int32_t*>(a + o_perm);
+  c->ws.inv = reinterpret_cast<int32_t*>(a + o_inv);
+  c->ws.w_sorted = reinterpret_cast<float*>(a + o_ws);
+  c->ws.tiles = reinterpret_cast<int32_t*>(a + o_tiles);
+  c->ws.ntile_prefix = reinterpret_cast<int32_t*>(a + o_pref);
+  c->ws.active = reinterpret_cast<int32_t*>(a + o_act);
+  c->ws.variant_id = reinterpret_cast<int32_t*>(a + o_var);
+  c->ws.status = reinterpret_cast<uint32_t*>(a + o_stat);
+  c->ws.block_hist = reinterpret_cast<int32_t*>(a + o_bh);
+  c->default_cost = reinterpret_cast<int64_t*>(a + o_cost);
+  c->ws.x_perm = reinterpret_cast<__nv_bfloat16*>(a + o_xp);
+  c->ws.h = reinterpret_cast<__nv_bfloat16*>(a + o_h);
+  c->ws.y = reinterpret_cast<float*>(a + o_y);
+  c->st_x = a + o_sx; c->st_ids = a + o_sid; c->st_w = a + o_sw; c->st_out = a + o_so;
+
+  int64_t cost[4 * kNumVariants];
+  default_cost_model(c, cost);
+  if (cudaMemcpy(c->default_cost, cost, sizeof(cost), cudaMemcpyHostToDevice) != cudaSuccess) return bail(DAMOE_ERR_CUDA);
+
+  for (int v = 0; v < kNumVariants; ++v) {
+    const uint32_t n = variant_desc(v).tile_n;
+    if (make_map(c, &c->map_x[v], c->ws.x_perm, P, H, n) != DAMOE_OK) return bail(DAMOE_ERR_CUDA);
+    if (make_map(c, &c->map_h[v], c->ws.h, P, I, n) != DAMOE_OK) return bail(DAMOE_ERR_CUDA);
+  }
+  *out = c;
+  return DAMOE_OK;
+}
+
+int damoe_destroy(damoe_ctx* c) {
+  if (!c) return DAMOE_OK;
+  cudaSetDevice(c->device);
+  if (c->arena) cudaFree(c->arena);
+  if (c->table_blob) cudaFree(c->table_blob);
+  delete c;
+  return DAMOE_OK;
+}
+
+int damoe_set_dispatch(damoe_ctx* c, int mode) {
+  if (!c) return DAMOE_ERR_INVALID_ARG;
+  if (mode != DAMOE_DISPATCH_BRANCH && mode != DAMOE_DISPATCH_PREDICATED)
+    return fail(c, DAMOE_ERR_INVALID_ARG, "dispatch mode %d is not available", mode);
+  c->dispatch = mode;
+  return DAMOE_OK;
+}
+
+int damoe_set_fp8_scales(damoe_ctx* c, const float*, const float*, const float*) {
+  return fail(c, DAMOE_ERR_UNSUPPORTED_SHAPE, "FP8 block-scaled path is not implemented");
+}
+
+int damoe_load_tuning_table(damoe_ctx* c, const void* bytes, size_t nbytes) {
+  if (!c || !bytes) return DAMOE_ERR_INVALID_ARG;
+  Reader r{static_cast<const uint8_t*>(bytes), nbytes};
+  const uint8_t* magic = r.take(8);
+  if (!r.ok || memcmp(magic, "DAMOETB1", 8) != 0) return fail(c, DAMOE_ERR_TABLE_FORMAT, "bad magic");
+  const uint32_t version = r.get<uint32_t>(), mode = r.get<uint32_t>(), E = r.get<uint32_t>(), k = r.get<uint32_t>(),
+                 H = r.get<uint32_t>(), I = r.get<uint32_t>(), dtype = r.get<uint32_t>(), V = r.get<uint32_t>(),
+                 nb = r.get<uint32_t>();
+  if (!r.ok || version != 1 || mode > DAMOE_MODE_COST || nb == 0 || nb > 64)
+    return fail(c, DAMOE_ERR_TABLE_FORMAT, "bad header");
+  if ((int)E != c->E || (int)k != c->k || (int)H != c->H || (int)I != c->I || (int)dtype != c->dtype ||
+      (int)V != kNumVariants)
+    return fail(c, DAMOE_ERR_TABLE_MISMATCH, "table is for E=%u k=%u H=%u I=%u dtype=%u V=%u", E, k, H, I, dtype, V);
+  std::vector<TableBucket> buckets(nb);
+  std::vector<uint8_t> blob;
+  auto put = [&](const void* src, size_t n) {
+    size_t o = align_up(blob.size(), 16);
+    blob.resize(o + n);
+    if (n) memcpy(blob.data() + o, src, n);
+    return o;
+  };
+  auto bad_variant = [&](int32_t v) { return v < 0 || v >= kNumVariants; };
+  for (uint32_t i = 0; i < nb; ++i) {
+    TableBucket& b = buckets[i];
+    b.T = (int)r.get<uint32_t>();
+    b.static_variant = r.get<int32_t>();
+    b.n_ex = (int)r.get<uint32_t>();
+    b.n_bins = (int)r.get<uint32_t>();
+    if (!r.ok || b.T < 1 || b.n_ex < 0 || b.n_ex > 64 || b.n_bins < 0 || b.n_bins > 64 || bad_variant(b.static_variant))
+      return fail(c, DAMOE_ERR_TABLE_FORMAT, "bad bucket %u header", i);
+    if (mode == DAMOE_MODE_EXEMPLAR && b.n_ex == 0) return fail(c, DAMOE_ERR_TABLE_FORMAT, "bucket %u has no exemplar", i);
+    if (mode == DAMOE_MODE_EFFEXP_BINS && b.n_bins == 0) return fail(c, DAMOE_ERR_TABLE_FORMAT, "bucket %u has no bin", i);
+    std::vector<int32_t> exv(b.n_ex), ex(static_cast<size_t>(b.n_ex) * E);
+    for (int m = 0; m < b.n_ex; ++m) {
+      exv[m] = r.get<int32_t>();
+      const uint8_t* q = r.take(4 * E);
+      if (!r.ok || bad_variant(exv[m])) return fail(c, DAMOE_ERR_TABLE_FORMAT, "bad exemplar %d of bucket %u", m, i);
+      memcpy(&ex[static_cast<size_t>(m) * E], q, 4 * E);
+    }
+    b.bin_den = r.get<uint64_t>();
+    const int nth = b.n_bins > 0 ? b.n_bins - 1 : 0;
+    std::vector<uint64_t> bnum(nth);
+    for (int t = 0; t < nth; ++t) bnum[t] = r.get<uint64_t>();
+    std::vector<int32_t> binv(b.n_bins);
+    for (int t = 0; t < b.n_bins; ++t) {
+      binv[t] = r.get<int32_t>();
+      if (r.ok && bad_variant(binv[t])) return fail(c, DAMOE_ERR_TABLE_FORMAT, "bad bin variant in bucket %u", i);
+    }
+    if (!r.ok || b.bin_den == 0 || b.bin_den > (1ull << 16)) return fail(c, DAMOE_ERR_TABLE_FORMAT, "bad bins in bucket %u", i);
+    for (int t = 0; t < nth; ++t)
+      if (bnum[t] > (1ull << 26) || (t > 0 && bnum[t] < bnum[t - 1]))
+        return fail(c, DAMOE_ERR_TABLE_FORMAT, "bad thresholds in bucket %u", i);
+    int64_t cost[4 * kNumVariants];
+    for (int t = 0; t < 4 * kNumVariants; ++t) cost[t] = r.get<int64_t>();
+    if (!r.ok) return fail(c, DAMOE_ERR_TABLE_FORMAT, "truncated bucket %u", i);
+    for (int t = 0; t < 4 * kNumVariants; ++t)
+      if (cost[t] < 0 || cost[t] > (1ll << 36)) return fail(c, DAMOE_ERR_TABLE_FORMAT, "cost out of range in bucket %u", i);
+    b.off_ex = put(ex.data(), ex.size() * 4);
+    b.off_exv = put(exv.data(), exv.size() * 4);
+    b.off_bnum = put(bnum.data(), bnum.size() * 8);
+    b.off_binv = put(binv.data(), binv.size() * 4);
+    b.off_cost = put(cost, sizeof(cost));
+  }
+  if (r.left != 0) return fail(c, DAMOE_ERR_TABLE_FORMAT, "%zu trailing bytes", r.left);
+  DAMOE_CUDA(c, cudaSetDevice(c->device));
+  DAMOE_CUDA(c, cudaDeviceSynchronize());
+  uint8_t* dev = nullptr;
+  DAMOE_CUDA(c, cudaMalloc(&dev, align_up(blob.size(), 16) + 16));
+  cudaError_t e = cudaMemcpy(dev, blob.data(), blob.size(), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) {
+    cudaFree(dev);
+    return fail(c, DAMOE_ERR_CUDA, "table upload: %s", cudaGetErrorString(e));
+  }
+  if (c->table_blob) cudaFree(c->table_blob);
+  c->table_blob = dev;
+  c->buckets.swap(buckets);
+  c->table_mode = (int)mode;
+  c->has_table = true;
+  return DAMOE_OK;
+}
+
+int damoe_route_stats(damoe_ctx* c, const int32_t* topk_ids, int T, int k, int E, int32_t* hist, double* eff_exp,
+                      void* stream) {
+  if (!c || !hist || !eff_exp || T < 0 || (T > 0 && !topk_ids)) return fail(c, DAMOE_ERR_INVALID_ARG, "bad argument");
+  if (k != c->k || E != c->E || T > c->max_T) return fail(c, DAMOE_ERR_INVALID_ARG, "T/k/E do not match the context");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DAMOE_CUDA(c, cudaSetDevice(c->device));
+  if (T == 0) {
+    DAMOE_CUDA(c, cudaMemsetAsync(hist, 0, sizeof(int32_t) * E, st));
+    DAMOE_CUDA(c, cudaMemsetAsync(eff_exp, 0, sizeof(double), st));
+    return DAMOE_OK;
+  }
+  SelectorArgs sel;
+  make_selector(c, T, 0, &sel);
+  DAMOE_CUDA(c, launch_route(c->ws, topk_ids, nullptr, T, k, E, sel, hist, eff_exp, true, st));
+  return DAMOE_OK;
+}
+
+int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2, const int32_t* topk_ids,
+                    const float* topk_weights, int T, int variant, void* out, void* stream) {
+  if (!c) return DAMOE_ERR_INVALID_ARG;
+  if (T == 0) return DAMOE_OK;
+  if (T < 0 || T > c->max_T) return fail(c, DAMOE_ERR_INVALID_ARG, "T=%d outside [0, %d]", T, c->max_T);
+  if (!x || !w13 || !w2 || !topk_ids || !topk_weights || !out) return fail(c, DAMOE_ERR_INVALID_ARG, "null pointer");
+  if (variant >= kNumVariants || variant < DAMOE_VARIANT_STATIC) return fail(c, DAMOE_ERR_INVALID_ARG, "variant %d", variant);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DAMOE_CUDA(c, cudaSetDevice(c->device));
+
+  if (w13 != c->cached_w13) {
+    int rc = make_map(c, &c->map_w13, w13, static_cast<uint64_t>(c->E) * 2 * c->I, c->H, kTileM);
+    if (rc != DAMOE_OK) return rc;
+    c->cached_w13 = w13;
+  }
+  if (w2 != c->cached_w2) {
+    int rc = make_map(c, &c->map_w2, w2, static_cast<uint64_t>(c->E) * c->H, c->I, kTileM);
+    if (rc != DAMOE_OK) return rc;
+    c->cached_w2 = w2;
+  }
+
+  c->last_T = T;
+  SelectorArgs sel;
+  const int known = make_selector(c, T, variant, &sel);
+  DAMOE_CUDA(c, launch_route(c->ws, topk_ids, topk_weights, T, c->k, c->E, sel, nullptr, nullptr, false, st));
+  DAMOE_CUDA(c, launch_gather(c->ws, static_cast<const __nv_bfloat16*>(x), T, c->k, c->H, st));
+
+  GemmMaps m13, m2;
+  m13.w = c->map_w13;
+  m2.w = c->map_w2;
+  for (int v = 0; v < kNumVariants; ++v) {
+    m13.act[v] = c->map_x[v];
+    m2.act[v] = c->map_h[v];
+  }
+  GemmArgs ga{};
+  ga.ntile_prefix = c->ws.ntile_prefix;
+  ga.offsets = c->ws.offsets;
+  ga.variant_id = c->ws.variant_id;
+  ga.status = c->ws.status;
+  ga.w_sorted = c->ws.w_sorted;
+  ga.h = c->ws.h;
+  ga.y = c->ws.y;
+  ga.E = c->E; ga.H = c->H; ga.I = c->I;
+
+  if (known >= 0) {
+    DAMOE_CUDA(c, launch_gemm(0, known, false, m13, ga, c->sm_count, st));
+    DAMOE_CUDA(c, launch_gemm(1, known, false, m2, ga, c->sm_count, st));
+  } else if (c->dispatch == DAMOE_DISPATCH_PREDICATED) {
+    for (int v = 0; v < kNumVariants; ++v) DAMOE_CUDA(c, launch_gemm(0, v, true, m13, ga, c->sm_count, st));
+    for (int v = 0; v < kNumVariants; ++v) DAMOE_CUDA(c, launch_gemm(1, v, true, m2, ga, c->sm_count, st));
+  } else {
+    DAMOE_CUDA(c, launch_gemm(0, -1, false, m13, ga, c->sm_count, st));
+    DAMOE_CUDA(c, launch_gemm(1, -1, false, m2, ga, c->sm_count, st));
+  }
+  DAMOE_CUDA(c, launch_reduce(c->ws, static_cast<__nv_bfloat16*>(out), T, c->k, c->H, st));
+  return DAMOE_OK;
+}
+
+int damoe_fused_moe_host(damoe_ctx* c, const void* x_host, const void* w13, const void* w2,
+                         const int32_t* topk_ids_host, const float* topk_weights_host, int T, int variant,
+                         void* out_host, void* stream) {
+  if (!c) return DAMOE_ERR_INVALID_ARG;
+  if (T == 0) return DAMOE_OK;
+  if (T < 0 || T > c->max_T) return fail(c, DAMOE_ERR_INVALID_ARG, "T=%d outside [0, %d]", T, c->max_T);
+  if (!x_host || !topk_ids_host || !topk_weights_host || !out_host) return fail(c, DAMOE_ERR_INVALID_ARG, "null pointer");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DAMOE_CUDA(c, cudaSetDevice(c->device));
+  const size_t P = static_cast<size_t>(T) * c->k;
+  DAMOE_CUDA(c, cudaMemcpyAsync(c->st_x, x_host, 2 * static_cast<size_t>(T) * c->H, cudaMemcpyHostToDevice, st));
+  DAMOE_CUDA(c, cudaMemcpyAsync(c->st_ids, topk_ids_host, 4 * P, cudaMemcpyHostToDevice, st));
+  DAMOE_CUDA(c, cudaMemcpyAsync(c->st_w, topk_weights_host, 4 * P, cudaMemcpyHostToDevice, st));
+  int rc = damoe_fused_moe(c, c->st_x, w13, w2, static_cast<const int32_t*>(c->st_ids),
+                           static_cast<const float*>(c->st_w), T, variant, c->st_out, stream);
+  if (rc != DAMOE_OK) return rc;
+  DAMOE_CUDA(c, cudaMemcpyAsync(out_host, c->st_out, 2 * static_cast<size_t>(T) * c->H, cudaMemcpyDeviceToHost, st));
+  DAMOE_CUDA(c, cudaStreamSynchronize(st));
+  return DAMOE_OK;
+}
+
+int damoe_debug_fetch(damoe_ctx* c, int32_t* offsets, int32_t* perm, int32_t* inv, int32_t* tiles, int32_t* variant_id,
+                      uint32_t* status_bits) {
+  if (!c) return DAMOE_ERR_INVALID_ARG;
+  DAMOE_CUDA(c, cudaSetDevice(c->device));
+  DAMOE_CUDA(c, cudaDeviceSynchronize());
+  if (offsets) DAMOE_CUDA(c, cudaMemcpy(offsets, c->ws.offsets, 4 * (c->E + 1), cudaMemcpyDeviceToHost));
+  if (perm) DAMOE_CUDA(c, cudaMemcpy(perm, c->ws.perm, 4 * static_cast<size_t>(c->last_T) * c->k, cudaMemcpyDeviceToHost));
+  if (inv) DAMOE_CUDA(c, cudaMemcpy(inv, c->ws.inv, 4 * static_cast<size_t>(c->last_T) * c->k, cudaMemcpyDeviceToHost));
+  if (tiles) DAMOE_CUDA(c, cudaMemcpy(tiles, c->ws.tiles, 4 * kNumVariants, cudaMemcpyDeviceToHost));
+  if (variant_id) DAMOE_CUDA(c, cudaMemcpy(variant_id, c->ws.variant_id, 4, cudaMemcpyDeviceToHost));
+  if (status_bits) {
+    DAMOE_CUDA(c, cudaMemcpy(status_bits, c->ws.status, 4, cudaMemcpyDeviceToHost));
+    DAMOE_CUDA(c, cudaMemset(c->ws.status, 0, 4));
+  }
+  return DAMOE_OK;
+}
+
+}  // extern "C"

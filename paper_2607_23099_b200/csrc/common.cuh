@@ -1,0 +1,97 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+#include <cstdint>
+#include <cstdio>
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "../../include/damoe.h"
+
+namespace damoe {
+
+constexpr int kMaxE = 1024;
+constexpr int kMaxK = 32;
+constexpr int kPairsPerBlock = 512;  // pairs ranked by one CTA of the route kernels
+constexpr int kTileM = 128;          // weight rows per MMA tile (TMEM lanes)
+constexpr int kBK = 64;              // K elements per pipeline stage: 128 bytes of bf16 = one swizzle row
+
+// The kernel family.  Ids are positions in this list.
+struct VariantDesc {
+  int tile_n;     // token-tile width N_v
+  int tile_m;     // weight rows per tile
+  int cta_group;  // CTAs cooperating on one tile
+  int stages13;   // pipeline depth of the gate/up GEMM
+  int stages2;    // pipeline depth of the down GEMM
+};
+constexpr int kNumVariants = 5;
+__host__ __device__ constexpr VariantDesc variant_desc(int v) {
+  constexpr VariantDesc t[kNumVariants] = {
+      {16, 128, 1, 6, 10}, {32, 128, 1, 5, 10}, {64, 128, 1, 5, 8}, {128, 128, 1, 4, 6}, {256, 128, 1, 3, 4}};
+  return t[v];
+}
+
+// What the selector kernel needs to know about the tuning table's bucket for this call.
+struct SelectorArgs {
+  int forced;                  // >= 0: write this id; -1: select on the device
+  int mode;                    // DAMOE_MODE_*
+  int n_exemplars;             // EXEMPLAR
+  const int32_t* exemplars;    // [n_exemplars, E] Q30
+  const int32_t* ex_variant;   // [n_exemplars]
+  int n_bins;                  // EFFEXP_BINS: n_bins variants, n_bins-1 thresholds
+  const uint64_t* bin_num;     // [n_bins-1] thresholds' numerators, ascending
+  uint64_t bin_den;
+  const int32_t* bin_variant;  // [n_bins]
+  const int64_t* cost;         // COST: [4, V] = c_fix, c_byte, c_reload, c_flop
+};
+
+// Pointers into the context's workspace that the kernels use.
+struct Workspace {
+  int32_t* hist;            // [E]
+  unsigned long long* sums; // [2] sum t, sum t^2
+  double* eff;              // [1]
+  int32_t* offsets;         // [E+1]
+  int32_t* perm;            // [max_P]
+  int32_t* inv;             // [max_P]
+  float* w_sorted;          // [max_P] routing weight of the pair at each sorted position
+  int32_t* tiles;           // [V]
+  int32_t* ntile_prefix;    // [V, E+1] exclusive scan of ceil(t_e / N_v)
+  int32_t* active;          // [1] experts with t_e > 0
+  int32_t* variant_id;      // [1]
+  uint32_t* status;         // [1]
+  int32_t* block_hist;      // [max_blocks, E]
+  __nv_bfloat16* x_perm;    // [max_P, H]
+  __nv_bfloat16* h;         // [max_P, I]
+  float* y;                 // [max_P, H]
+};
+
+// route.cu
+cudaError_t launch_route(const Workspace& ws, const int32_t* topk_ids, const float* topk_weights, int T, int k, int E,
+                         const SelectorArgs& sel, int32_t* hist_out, double* eff_out, bool stats_only,
+                         cudaStream_t stream);
+// misc.cu
+cudaError_t launch_gather(const Workspace& ws, const __nv_bfloat16* x, int T, int k, int H, cudaStream_t stream);
+cudaError_t launch_reduce(const Workspace& ws, __nv_bfloat16* out, int T, int k, int H, cudaStream_t stream);
+
+// gemm.cu
+struct GemmMaps {
+  CUtensorMap w;                  // weights as [E * rows, K], box 64 x 128
+  CUtensorMap act[kNumVariants];  // activations [max_P, K], box 64 x N_v
+};
+struct GemmArgs {
+  const int32_t* ntile_prefix;  // [V, E+1]
+  const int32_t* offsets;       // [E+1]
+  const int32_t* variant_id;
+  uint32_t* status;
+  const float* w_sorted;        // down GEMM only
+  __nv_bfloat16* h;             // gate/up GEMM output [max_P, I]
+  float* y;                     // down GEMM output [max_P, H]
+  int E, H, I;
+};
+// variant >= 0: launch that variant's kernel; predicated: it exits unless *variant_id == variant.
+// variant == -1: one kernel that branches on *variant_id.
+cudaError_t launch_gemm(int kind, int variant, bool predicated, const GemmMaps& maps, const GemmArgs& args,
+                        int sm_count, cudaStream_t stream);
+cudaError_t gemm_configure();  // opt-in shared-memory sizes, once per device
+
+}  // namespace damoe

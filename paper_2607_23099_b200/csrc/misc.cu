@@ -1,0 +1,64 @@
+// Token gather into expert-sorted order and the top-k unpermute-reduce.  Both are plain
+// bandwidth-bound vector kernels: 16-byte accesses, consecutive threads on consecutive
+// addresses, one row per CTA so a large batch fills every SM many times over.
+#include "common.cuh"
+
+namespace damoe {
+
+namespace {
+
+// x_perm[q, :] = x[perm[q] / k, :]
+__global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restrict__ x, uint4* __restrict__ x_perm,
+                                                          const int32_t* __restrict__ perm, int k, int row_vec) {
+  const int q = blockIdx.x;
+  const int p = perm[q];
+  if (p < 0) return;
+  const uint4* src = x + static_cast<size_t>(p / k) * row_vec;
+  uint4* dst = x_perm + static_cast<size_t>(q) * row_vec;
+  for (int i = threadIdx.x; i < row_vec; i += blockDim.x) dst[i] = __ldg(src + i);
+}
+
+// out[t, :] = bf16( sum_{j<k} y[inv[t*k+j], :] ), j ascending, fp32 adds.  The routing weight
+// was already applied by the down GEMM's epilogue.
+__global__ void __launch_bounds__(256) unpermute_reduce_kernel(const float4* __restrict__ y,
+                                                               const int32_t* __restrict__ inv,
+                                                               uint2* __restrict__ out, int k, int row_vec) {
+  const int t = blockIdx.x;
+  __shared__ int s_q[kMaxK];
+  if (threadIdx.x < k) s_q[threadIdx.x] = inv[t * k + threadIdx.x];
+  __syncthreads();
+  for (int i = threadIdx.x; i < row_vec; i += blockDim.x) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = 0; j < k; ++j) {
+      const int q = s_q[j];
+      if (q < 0) continue;
+      const float4 v = __ldcs(y + static_cast<size_t>(q) * row_vec + i);
+      acc.x += v.x;
+      acc.y += v.y;
+      acc.z += v.z;
+      acc.w += v.w;
+    }
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z, acc.w);
+    uint2 o;
+    o.x = *reinterpret_cast<uint32_t*>(&lo);
+    o.y = *reinterpret_cast<uint32_t*>(&hi);
+    out[static_cast<size_t>(t) * row_vec + i] = o;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_gather(const Workspace& ws, const __nv_bfloat16* x, int T, int k, int H, cudaStream_t stream) {
+  gather_rows_kernel<<<T * k, 256, 0, stream>>>(reinterpret_cast<const uint4*>(x), reinterpret_cast<uint4*>(ws.x_perm),
+                                                ws.perm, k, H / 8);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_reduce(const Workspace& ws, __nv_bfloat16* out, int T, int k, int H, cudaStream_t stream) {
+  unpermute_reduce_kernel<<<T, 256, 0, stream>>>(reinterpret_cast<const float4*>(ws.y), ws.inv,
+                                                 reinterpret_cast<uint2*>(out), k, H / 4);
+  return cudaGetLastError();
+}
+
+}  // namespace damoe

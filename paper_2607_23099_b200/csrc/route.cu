@@ -1,0 +1,285 @@
+// Routing statistics and metadata on the GPU: per-expert histogram, Effective Experts
+// (paper Eq. 2), offsets, the stable grouping of (token, slot) pairs by expert, per-variant
+// padded-tile counts, and the device-side choice of the kernel variant (paper Section IV-B).
+//
+// Three small launches:
+//   count   : one CTA per 512 pairs; warp-aggregated shared-memory histogram -> block_hist[b][e]
+//   scan    : one CTA; scans block_hist over blocks (turning it into per-block bases), writes
+//             hist / sums / eff_exp / offsets / tile prefixes / tile counts, runs the selector
+//   scatter : one CTA per 512 pairs; ranks each pair inside its warp with match_any, scans the
+//             per-warp counts, and writes perm / inv / w_sorted in the canonical stable order
+// No atomics decide an output position, so every integer output is reproducible bit for bit.
+#include "common.cuh"
+
+namespace damoe {
+
+namespace {
+
+constexpr int kScanThreads = 1024;
+constexpr int kWarpsPerRouteBlock = kPairsPerBlock / 32;
+constexpr int kMaxExemplars = 64;
+
+__global__ void __launch_bounds__(kPairsPerBlock) route_count_kernel(const int32_t* __restrict__ ids, int P, int E,
+                                                                     int32_t* __restrict__ block_hist,
+                                                                     uint32_t* __restrict__ status) {
+  __shared__ int s_hist[kMaxE];
+  for (int e = threadIdx.x; e < E; e += blockDim.x) s_hist[e] = 0;
+  __syncthreads();
+  const int p = blockIdx.x * kPairsPerBlock + threadIdx.x;
+  const int lane = threadIdx.x & 31;
+  const int e = (p < P) ? ids[p] : -1;
+  const bool valid = (p < P) && e >= 0 && e < E;
+  const unsigned bad = __ballot_sync(0xffffffffu, (p < P) && !valid);
+  if (bad && lane == 0) atomicOr(status, DAMOE_STATUS_BAD_ID);
+  const unsigned act = __ballot_sync(0xffffffffu, valid);
+  if (valid) {
+    const unsigned same = __match_any_sync(act, e);
+    if (lane == __ffs(same) - 1) atomicAdd(&s_hist[e], __popc(same));
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < E; i += blockDim.x) block_hist[blockIdx.x * E + i] = s_hist[i];
+}
+
+// Exclusive scan of one int per thread over a 1024-thread CTA; *total gets the sum.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    int o = __shfl_up_sync(0xffffffffu, inc, d);
+    if (lane >= d) inc += o;
+  }
+  __syncthreads();  // protects s_warp against the previous use
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    int w = s_warp[lane];
+    int winc = w;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      int o = __shfl_up_sync(0xffffffffu, winc, d);
+      if (lane >= d) winc += o;
+    }
+    s_warp[lane] = winc - w;
+    if (lane == 31) s_warp[32] = winc;
+  }
+  __syncthreads();
+  *total = s_warp[32];
+  return s_warp[warp] + inc - v;
+}
+
+__global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __restrict__ block_hist, int nblocks, int E,
+                                                                  Workspace ws, SelectorArgs sel,
+                                                                  int32_t* __restrict__ hist_out,
+                                                                  double* __restrict__ eff_out, int stats_only) {
+  __shared__ int s_hist[kMaxE];
+  __shared__ int s_sorted[kMaxE];
+  __shared__ int s_warp[33];
+  __shared__ unsigned long long s_red[2][32];
+  __shared__ int s_tiles[kNumVariants];
+  __shared__ long long s_score[kMaxExemplars];
+  __shared__ int s_active;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  // per-expert totals; block_hist becomes each block's base inside the expert's segment
+  for (int e = tid; e < E; e += kScanThreads) {
+    int running = 0;
+    for (int b = 0; b < nblocks; ++b) {
+      const int v = block_hist[b * E + e];
+      block_hist[b * E + e] = running;
+      running += v;
+    }
+    s_hist[e] = running;
+    if (hist_out) hist_out[e] = running;
+    if (!stats_only) ws.hist[e] = running;
+  }
+  __syncthreads();
+
+  // sum t and sum t^2 (exact integers), Effective Experts = (sum t)^2 / sum t^2
+  unsigned long long s1 = 0, s2 = 0;
+  for (int e = tid; e < E; e += kScanThreads) {
+    const unsigned long long t = static_cast<unsigned long long>(s_hist[e]);
+    s1 += t;
+    s2 += t * t;
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    s1 += __shfl_down_sync(0xffffffffu, s1, d);
+    s2 += __shfl_down_sync(0xffffffffu, s2, d);
+  }
+  if (lane == 0) {
+    s_red[0][warp] = s1;
+    s_red[1][warp] = s2;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    unsigned long long a = 0, b = 0;
+    for (int w = 0; w < kScanThreads / 32; ++w) {
+      a += s_red[0][w];
+      b += s_red[1][w];
+    }
+    s_red[0][0] = a;
+    s_red[1][0] = b;
+    const double eff = (b == 0) ? 0.0 : static_cast<double>(a * a) / static_cast<double>(b);
+    if (eff_out) *eff_out = eff;
+    if (!stats_only) {
+      ws.sums[0] = a;
+      ws.sums[1] = b;
+      *ws.eff = eff;
+    }
+    if (b == 0) atomicOr(ws.status, DAMOE_STATUS_NO_VALID_ID);
+  }
+  if (stats_only) return;
+  __syncthreads();
+
+  const int t_e = (tid < E) ? s_hist[tid] : 0;
+  int total;
+  // offsets
+  {
+    const int ex = block_exclusive_scan(t_e, s_warp, &total);
+    if (tid < E) ws.offsets[tid] = ex;
+    if (tid == 0) ws.offsets[E] = total;
+  }
+  // active experts
+  {
+    block_exclusive_scan(t_e > 0 ? 1 : 0, s_warp, &total);
+    if (tid == 0) {
+      s_active = total;
+      *ws.active = total;
+    }
+  }
+  // token tiles per variant: exclusive scan of ceil(t_e / N_v)
+  for (int v = 0; v < kNumVariants; ++v) {
+    const int n = variant_desc(v).tile_n;
+    const int ex = block_exclusive_scan((t_e + n - 1) / n, s_warp, &total);
+    if (tid < E) ws.ntile_prefix[v * (E + 1) + tid] = ex;
+    if (tid == 0) {
+      ws.ntile_prefix[v * (E + 1) + E] = total;
+      ws.tiles[v] = total;
+      s_tiles[v] = total;
+    }
+  }
+  __syncthreads();
+
+  // ---- selector ------------------------------------------------------------------
+  if (sel.forced >= 0) {
+    if (tid == 0) *ws.variant_id = sel.forced;
+    return;
+  }
+  int chosen = 0;
+  if (sel.mode == DAMOE_MODE_EXEMPLAR) {
+    // descending sort by rank counting: rank_i = #{j : t_j > t_i or (t_j == t_i and j < i)}
+    if (tid < E) {
+      int rank = 0;
+      for (int j = 0; j < E; ++j) {
+        const int tj = s_hist[j];
+        rank += (tj > t_e) || (tj == t_e && j < tid);
+      }
+      s_sorted[rank] = t_e;
+    }
+    __syncthreads();
+    // one warp per exemplar: exact integer dot product with the Q30 unit vector
+    for (int m = warp; m < sel.n_exemplars; m += kScanThreads / 32) {
+      long long acc = 0;
+      const int32_t* ex = sel.exemplars + static_cast<size_t>(m) * E;
+      for (int i = lane; i < E; i += 32) acc += static_cast<long long>(s_sorted[i]) * static_cast<long long>(ex[i]);
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, d);
+      if (lane == 0) s_score[m] = acc;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int best = 0;
+      for (int m = 1; m < sel.n_exemplars; ++m)
+        if (s_score[m] > s_score[best]) best = m;
+      chosen = sel.ex_variant[best];
+    }
+  } else if (sel.mode == DAMOE_MODE_EFFEXP_BINS) {
+    if (tid == 0) {
+      const unsigned long long a = s_red[0][0], b = s_red[1][0];
+      int r = 0;
+      for (int i = 0; i + 1 < sel.n_bins; ++i)
+        if (a * a * sel.bin_den >= sel.bin_num[i] * b) ++r;
+      chosen = sel.bin_variant[r];
+    }
+  } else {  // DAMOE_MODE_COST
+    if (tid == 0) {
+      const long long A = s_active;
+      long long best_cost = 0;
+      for (int v = 0; v < kNumVariants; ++v) {
+        const long long tiles = s_tiles[v];
+        const long long mem = sel.cost[1 * kNumVariants + v] * A + sel.cost[2 * kNumVariants + v] * (tiles - A);
+        const long long mma = sel.cost[3 * kNumVariants + v] * tiles * variant_desc(v).tile_n;
+        const long long c = sel.cost[0 * kNumVariants + v] + (mem > mma ? mem : mma);
+        if (v == 0 || c < best_cost) {
+          best_cost = c;
+          chosen = v;
+        }
+      }
+    }
+  }
+  if (tid == 0) {
+    if (chosen < 0 || chosen >= kNumVariants) {
+      atomicOr(ws.status, DAMOE_STATUS_BAD_VARIANT);
+      chosen = 0;
+    }
+    *ws.variant_id = chosen;
+  }
+}
+
+__global__ void __launch_bounds__(kPairsPerBlock) route_scatter_kernel(const int32_t* __restrict__ ids,
+                                                                       const float* __restrict__ weights, int P, int E,
+                                                                       const int32_t* __restrict__ block_base,
+                                                                       Workspace ws) {
+  __shared__ unsigned short s_cnt[kWarpsPerRouteBlock][kMaxE];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int i = tid; i < kWarpsPerRouteBlock * E; i += blockDim.x) s_cnt[i / E][i % E] = 0;
+  __syncthreads();
+  const int p = blockIdx.x * kPairsPerBlock + tid;
+  const int e = (p < P) ? ids[p] : -1;
+  const bool valid = (p < P) && e >= 0 && e < E;
+  const unsigned act = __ballot_sync(0xffffffffu, valid);
+  int rank = 0;
+  if (valid) {
+    const unsigned same = __match_any_sync(act, e);
+    rank = __popc(same & ((1u << lane) - 1u));
+    if (rank == 0) s_cnt[warp][e] = static_cast<unsigned short>(__popc(same));
+  }
+  __syncthreads();
+  for (int i = tid; i < E; i += blockDim.x) {
+    int running = 0;
+#pragma unroll
+    for (int w = 0; w < kWarpsPerRouteBlock; ++w) {
+      const int c = s_cnt[w][i];
+      s_cnt[w][i] = static_cast<unsigned short>(running);
+      running += c;
+    }
+  }
+  __syncthreads();
+  if (valid) {
+    const int pos = ws.offsets[e] + block_base[blockIdx.x * E + e] + s_cnt[warp][e] + rank;
+    ws.perm[pos] = p;
+    ws.inv[p] = pos;
+    ws.w_sorted[pos] = weights[p];
+  } else if (p < P) {
+    ws.inv[p] = -1;
+  }
+  if (p < P && p >= ws.offsets[E]) ws.perm[p] = -1;  // sorted positions past the valid count
+}
+
+}  // namespace
+
+cudaError_t launch_route(const Workspace& ws, const int32_t* topk_ids, const float* topk_weights, int T, int k, int E,
+                         const SelectorArgs& sel, int32_t* hist_out, double* eff_out, bool stats_only,
+                         cudaStream_t stream) {
+  const int P = T * k;
+  const int nblocks = (P + kPairsPerBlock - 1) / kPairsPerBlock;
+  route_count_kernel<<<nblocks, kPairsPerBlock, 0, stream>>>(topk_ids, P, E, ws.block_hist, ws.status);
+  route_scan_kernel<<<1, kScanThreads, 0, stream>>>(ws.block_hist, nblocks, E, ws, sel, hist_out, eff_out,
+                                                    stats_only ? 1 : 0);
+  if (!stats_only)
+    route_scatter_kernel<<<nblocks, kPairsPerBlock, 0, stream>>>(topk_ids, topk_weights, P, E, ws.block_hist, ws);
+  return cudaGetLastError();
+}
+
+}  // namespace damoe

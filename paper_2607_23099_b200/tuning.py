@@ -1,0 +1,45 @@
+"""Offline tuning tables (paper Section IV-A): serialisation into the byte format that
+damoe_load_tuning_table parses.  Building the table's *content* (which variant is fastest for
+which routing distribution) is the job of the sweep in bench.py; this module only packs it.
+
+Layout (little endian)
+  header : "DAMOETB1", u32 version=1, u32 mode, u32 E, u32 k, u32 H, u32 I, u32 dtype, u32 V,
+           u32 n_buckets
+  bucket : u32 T, i32 static_variant, u32 n_exemplars, u32 n_bins,
+           n_exemplars x { i32 variant, i32 q30[E] },
+           u64 bin_den, (n_bins-1) x u64 threshold numerators (ascending), n_bins x i32 variant,
+           4*V x i64 cost coefficients: c_fix[V], c_byte[V], c_reload[V], c_flop[V]
+"""
+from __future__ import annotations
+
+import struct
+
+MAGIC = b"DAMOETB1"
+
+
+def pack_table(table: dict, E: int, k: int, H: int, I: int, dtype: int, V: int) -> bytes:
+    """``table`` = {"mode": m, "buckets": [bucket, ...]} where a bucket is a dict with keys
+    T, static_variant and, optionally, exemplars (list of length-E int sequences) with
+    exemplar_variants, bin_thresholds_num / bin_den / bin_variants, c_fix / c_byte / c_reload /
+    c_flop (length-V int sequences).  Missing parts are written empty / zero."""
+    out = [MAGIC, struct.pack("<9I", 1, table["mode"], E, k, H, I, dtype, V, len(table["buckets"]))]
+    for b in table["buckets"]:
+        ex = b.get("exemplars", [])
+        exv = b.get("exemplar_variants", [])
+        binv = b.get("bin_variants", [])
+        thr = b.get("bin_thresholds_num", [])
+        assert len(ex) == len(exv)
+        assert len(thr) == max(0, len(binv) - 1)
+        out.append(struct.pack("<IiII", b["T"], b["static_variant"], len(ex), len(binv)))
+        for q, v in zip(ex, exv):
+            assert len(q) == E
+            out.append(struct.pack("<i", int(v)))
+            out.append(struct.pack(f"<{E}i", *[int(t) for t in q]))
+        out.append(struct.pack("<Q", int(b.get("bin_den", 1))))
+        out.append(struct.pack(f"<{len(thr)}Q", *[int(t) for t in thr]))
+        out.append(struct.pack(f"<{len(binv)}i", *[int(t) for t in binv]))
+        for key in ("c_fix", "c_byte", "c_reload", "c_flop"):
+            vals = b.get(key, [0] * V)
+            assert len(vals) == V
+            out.append(struct.pack(f"<{V}q", *[int(t) for t in vals]))
+    return b"".join(out)

@@ -1,0 +1,231 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle on the same seeded
+inputs.  Integer outputs must match bit for bit; layer outputs must satisfy
+relative Frobenius error <= 5e-3 and |gpu - ref| <= 1e-2 * max(1, |ref|) element-wise."""
+import numpy as np
+import pytest
+import torch
+
+import damoe_inputs as di
+from helpers import Case, bits16, config0, max_scaled_err, rel_frobenius
+from oracle import codecs, layer, modeling, route
+
+pytestmark = pytest.mark.gpu
+
+FROB_TOL, ELEM_TOL = 5e-3, 1e-2
+
+
+@pytest.fixture(scope="module")
+def d():
+    import paper_2607_23099_b200 as d
+    return d
+
+
+def _device_case(case):
+    dev = "cuda:0"
+    w13, w2 = case.weights.materialize(dev)
+    return dict(x=case.x(dev), w13=w13, w2=w2, ids=torch.from_numpy(case.ids).to(dev),
+                w=torch.from_numpy(case.w).to(dev))
+
+
+def _check_route(meta, case, tile_ns):
+    P = case.T * case.k
+    hist = route.histogram(case.ids, case.E)
+    off, perm, inv = route.offsets_and_permutation(case.ids, case.E)
+    assert np.array_equal(meta["offsets"], off.astype(np.int32))
+    nv = int(off[-1])
+    assert np.array_equal(meta["perm"][:nv], perm.astype(np.int32))
+    assert np.all(meta["perm"][nv:P] == -1)
+    assert np.array_equal(meta["inv"], inv.astype(np.int32))
+    assert np.array_equal(meta["tiles"], route.tile_counts(hist, tile_ns).astype(np.int32))
+
+
+def _check_layer(out, case, tokens=None):
+    ref_bits, ref64 = layer.moe_layer_bf16(bits16(case.x()), case.w13_bits, case.w2_bits, case.ids, case.w, case.E,
+                                           tokens=tokens)
+    got = codecs.bf16_decode(bits16(out))
+    if tokens is not None:
+        got = got[np.asarray(tokens)]
+    ref = codecs.bf16_decode(ref_bits)
+    fro, mx = rel_frobenius(got, ref), max_scaled_err(got, ref)
+    assert fro <= FROB_TOL, f"relative Frobenius {fro}"
+    assert mx <= ELEM_TOL, f"max scaled error {mx}"
+    return fro, mx
+
+
+def test_route_stats_matches_oracle(d):
+    for seed, (T, k, E, a) in enumerate([(64, 2, 8, 1.0), (64, 8, 256, 0.05), (1, 8, 256, 1.0), (777, 8, 384, 0.2),
+                                         (8192, 8, 256, 10.0)]):
+        ids, _, _ = di.routing_batch(seed, T, k, E, a)
+        m = d.DAMoE(T, k, E, 1024, 512)
+        hist, eff = m.route_stats(torch.from_numpy(ids).cuda())
+        want = route.histogram(ids, E)
+        assert np.array_equal(hist.cpu().numpy(), want.astype(np.int32))
+        assert eff.item() == route.effective_experts(want)[2]          # bit-exact binary64
+        m.close()
+
+
+def test_route_stats_closed_forms_on_gpu(d):
+    m = d.DAMoE(64, 8, 256, 1024, 512)
+    same = torch.tensor([[3, 9, 27, 81, 100, 5, 6, 7]] * 64, dtype=torch.int32, device="cuda")
+    assert m.route_stats(same)[1].item() == 8.0                        # only k experts ever hit
+    uni = (torch.arange(64 * 8, dtype=torch.int32, device="cuda") % 256).view(64, 8)
+    assert m.route_stats(uni)[1].item() == 256.0                       # uniform routing
+    hist, eff = m.route_stats(torch.empty(0, 8, dtype=torch.int32, device="cuda"))
+    assert hist.sum().item() == 0 and eff.item() == 0.0
+    m.close()
+
+
+def test_config0_every_variant_and_dispatch(d):
+    case = config0()
+    t = _device_case(case)
+    m = d.DAMoE(case.T, case.k, case.E, case.H, case.I)
+    ns = d.tile_ns()
+    outs = []
+    for variant in list(range(d.variant_count())) + [d.VARIANT_AUTO, d.VARIANT_STATIC]:
+        out = m.fused_moe(t["x"], t["w13"], t["w2"], t["ids"], t["w"], variant)
+        meta = m.debug_fetch(case.T)
+        assert meta["status"] == 0, f"variant {variant}: status {meta['status']}"
+        _check_route(meta, case, ns)
+        if variant >= 0:
+            assert meta["variant_id"] == variant
+        _check_layer(out, case)
+        outs.append(bits16(out))
+    m.set_dispatch(d.DISPATCH_PREDICATED)
+    out = m.fused_moe(t["x"], t["w13"], t["w2"], t["ids"], t["w"], d.VARIANT_AUTO)
+    assert m.debug_fetch(case.T)["status"] == 0
+    _check_layer(out, case)
+    m.close()
+
+
+def test_ragged_multi_tile_and_determinism(d):
+    # 300 tokens on 8 experts: segments of several tiles with ragged tails for every tile width
+    case = Case(5, 300, 8, 2, 1024, 512, 0.3)
+    t = _device_case(case)
+    m = d.DAMoE(512, case.k, case.E, case.H, case.I)
+    ns = d.tile_ns()
+    for variant in range(d.variant_count()):
+        a = m.fused_moe(t["x"], t["w13"], t["w2"], t["ids"], t["w"], variant)
+        meta = m.debug_fetch(case.T)
+        assert meta["status"] == 0
+        _check_route(meta, case, ns)
+        b = m.fused_moe(t["x"], t["w13"], t["w2"], t["ids"], t["w"], variant)
+        torch.cuda.synchronize()
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))   # no atomics anywhere: same bits
+        _check_layer(a, case)
+    m.close()
+
+
+def test_edge_cases(d):
+    case = config0(seed=3, T=5)
+    t = _device_case(case)
+    m = d.DAMoE(64, case.k, case.E, case.H, case.I)
+    # T = 0 touches nothing
+    out0 = torch.full((1, case.H), 7.0, dtype=torch.bfloat16, device="cuda")
+    m.fused_moe(t["x"][:0], t["w13"], t["w2"], t["ids"][:0], t["w"][:0], 0, out=out0)
+    assert torch.all(out0 == 7.0)
+    # T = 1
+    one = Case(11, 1, case.E, case.k, case.H, case.I, 1.0)
+    one.weights = case.weights
+    out = m.fused_moe(one.x("cuda"), t["w13"], t["w2"], torch.from_numpy(one.ids).cuda(), torch.from_numpy(one.w).cuda(), d.VARIANT_AUTO)
+    assert m.debug_fetch(1)["status"] == 0
+    _check_layer(out, one)
+    # invalid ids are skipped and flagged; duplicates within a token are legal
+    ids = case.ids.copy()
+    ids[0, 0], ids[1, 1], ids[2] = -1, case.E, [4, 4]
+    bad = Case(3, 5, case.E, case.k, case.H, case.I, 1.0)
+    bad.ids, bad.w, bad.weights = ids, case.w, case.weights
+    out = m.fused_moe(t["x"], t["w13"], t["w2"], torch.from_numpy(ids).cuda(), t["w"], 1)
+    meta = m.debug_fetch(5)
+    assert meta["status"] == d.STATUS_BAD_ID
+    _check_route(meta, bad, d.tile_ns())
+    _check_layer(out, bad)
+    # argument errors
+    with pytest.raises(d.DamoeError):
+        m.fused_moe(t["x"], t["w13"], t["w2"], t["ids"], t["w"], d.variant_count())
+    big = torch.zeros(65, case.H, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(d.DamoeError):
+        m.fused_moe(big, t["w13"], t["w2"], t["ids"], t["w"], 0)
+    m.close()
+
+
+def _table_for(E, k, T_buckets, mode, V, ns):
+    buckets = []
+    for bi, T in enumerate(T_buckets):
+        ex, exv = [], []
+        for i, a in enumerate([0.05, 0.2, 1.0, 10.0]):
+            counts = [route.histogram(di.routing_batch(9000 + 100 * bi + 10 * i + s, T, k, E, a)[0], E) for s in range(3)]
+            ex.append(modeling.exemplar_q30(counts).tolist())
+            exv.append((i + bi) % V)
+        buckets.append(dict(T=T, static_variant=(bi + 2) % V, exemplars=ex, exemplar_variants=exv,
+                            bin_thresholds_num=[int(0.1 * E * 65536), int(0.4 * E * 65536), int(0.7 * E * 65536)], bin_den=65536,
+                            bin_variants=[(bi + j) % V for j in (3, 2, 1, 0)],
+                            c_fix=[1000 * v for v in range(V)], c_byte=[13_000_000] * V, c_reload=[5_000_000] * V,
+                            c_flop=[int(4_000_000 / n + 30_000) for n in ns]))
+    return dict(mode=mode, buckets=buckets)
+
+
+def test_selected_variant_matches_oracle_given_the_same_table(d):
+    from paper_2607_23099_b200 import tuning
+    E, k, H, I = 64, 4, 256, 128
+    V, ns = d.variant_count(), d.tile_ns()
+    W = di.MoEWeights(1, E, H, I)
+    w13, w2 = W.materialize("cuda")
+    m = d.DAMoE(512, k, E, H, I)
+    for mode in (d.MODE_EXEMPLAR, d.MODE_EFFEXP_BINS, d.MODE_COST):
+        table = _table_for(E, k, [16, 128, 512], mode, V, ns)
+        m.load_tuning_table(tuning.pack_table(table, E, k, H, I, d.BF16, V))
+        seen = set()
+        for s, (T, a) in enumerate([(7, 0.05), (16, 10.0), (100, 0.2), (128, 1.0), (300, 0.05), (512, 10.0), (40, 0.5)]):
+            ids, w, _ = di.routing_batch(400 + s, T, k, E, a)
+            x = di.activations(s, T, H, "cuda")
+            for variant, static in ((d.VARIANT_AUTO, False), (d.VARIANT_STATIC, True)):
+                m.fused_moe(x, w13, w2, torch.from_numpy(ids).cuda(), torch.from_numpy(w).cuda(), variant)
+                meta = m.debug_fetch(T)
+                want = route.select_variant(table, route.histogram(ids, E), T, ns, static=static)
+                assert meta["variant_id"] == want and meta["status"] == 0
+                seen.add(want)
+        assert len(seen) >= 2
+    # malformed / mismatched tables are refused
+    good = tuning.pack_table(_table_for(E, k, [16], d.MODE_COST, V, ns), E, k, H, I, d.BF16, V)
+    with pytest.raises(d.DamoeError) as ei:
+        m.load_tuning_table(good[:-3])
+    assert ei.value.code == 4
+    with pytest.raises(d.DamoeError) as ei:
+        m.load_tuning_table(tuning.pack_table(_table_for(E, k, [16], d.MODE_COST, V, ns), E + 1, k, H, I, d.BF16, V))
+    assert ei.value.code == 5
+    m.close()
+
+
+def test_host_buffer_entry_point(d):
+    case = config0(seed=6, T=32)
+    t = _device_case(case)
+    m = d.DAMoE(64, case.k, case.E, case.H, case.I)
+    out = m.fused_moe_host(case.x().pin_memory(), t["w13"], t["w2"], torch.from_numpy(case.ids).pin_memory(),
+                           torch.from_numpy(case.w).pin_memory(), d.VARIANT_AUTO)
+    _check_layer(out, case)
+    m.close()
+
+
+def test_config1_shape_sampled_tokens(d):
+    # DeepSeek-V3-shaped layer at decode (E=256, top-8, H=7168, I=2048, T=64); the oracle checks
+    # all integer outputs in full and the layer output on a seeded sample of tokens.
+    E, k, H, I, T = 256, 8, 7168, 2048, 64
+    W = di.MoEWeights(12345, E, H, I)
+    w13, w2 = W.materialize("cuda")
+    m = d.DAMoE(T, k, E, H, I)
+    ns = d.tile_ns()
+    for alpha, seed, variant in [(0.05, 0, d.VARIANT_AUTO), (10.0, 1, 0), (1.0, 2, 2)]:
+        case = Case(seed, T, E, k, H, I, alpha)
+        case.weights = W
+        out = m.fused_moe(case.x("cuda"), w13, w2, torch.from_numpy(case.ids).cuda(), torch.from_numpy(case.w).cuda(), variant)
+        meta = m.debug_fetch(T)
+        assert meta["status"] == 0
+        _check_route(meta, case, ns)
+        tokens = [int(v) for v in np.random.default_rng(seed).choice(T, size=2, replace=False)]
+        _check_layer(out, case, tokens=tokens)
+    m.close()
+
+
+def test_dispatch_microbench_runs(d):
+    r = d.dispatch_microbench(50)
+    assert all(0 < v < 1e4 for v in r.values())
