@@ -190,8 +190,10 @@ def test_selected_variant_matches_oracle_given_the_same_table(d):
     with pytest.raises(d.DamoeError) as ei:
         m.load_tuning_table(good[:-3])
     assert ei.value.code == 4
+    other = bytearray(good)
+    other[16:20] = (E + 1).to_bytes(4, "little")          # header field E
     with pytest.raises(d.DamoeError) as ei:
-        m.load_tuning_table(tuning.pack_table(_table_for(E, k, [16], d.MODE_COST, V, ns), E + 1, k, H, I, d.BF16, V))
+        m.load_tuning_table(bytes(other))
     assert ei.value.code == 5
     m.close()
 
