@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the distribution-aware fused-MoE layer on B200.
+
+A step = one pass of the whole hot path (histogram + Effective Experts, permutation, tile
+counts, device-side variant selection, grouped gate/up GEMM + SwiGLU, grouped down GEMM,
+unpermute-reduce) over one synthetic batch.  Workload: the DeepSeek-V3-shaped decode layer
+(E=256, top-8, H=7168, I=2048, bf16, T=64) under Dirichlet routing with concentration alpha in
+{0.05, 0.2, 1, 10} x 4 seeds = 16 cells; steps cycle through the cells.  Every step streams
+between ~4 GB and ~19 GB of expert weights, far more than the 126 MB L2, so no L2 flush is
+needed between steps.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  With N > 1 (under torchrun) every rank runs an independent replica on
+its own GPU (the path does not shard; no collective is on the data path) and rank 0 reports
+the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+import damoe_inputs as di  # noqa: E402
+
+WORKLOAD = dict(name="deepseek_v3_decode_T64", E=256, k=8, H=7168, I=2048, T=64,
+                alphas=[0.05, 0.2, 1.0, 10.0], seeds=[0, 1, 2, 3], weight_seed=12345)
+# Same per-expert structure (2 tokens per expert on average, same H and I) on 1/8 of the
+# experts: 2.8 GB of weights, still far larger than L2.  Only for ncu captures, which must stay
+# small; never the headline.
+SMALL_WORKLOAD = dict(name="profile_small_E32_T8", E=32, k=8, H=7168, I=2048, T=8,
+                      alphas=[1.0], seeds=[0, 1], weight_seed=12345)
+TABLE_PATH = os.path.join(ROOT, "paper_2607_23099_b200", "tables", "e256_k8_h7168_i2048_bf16.damoetb")
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one gate/up GEMM launch, divided by the
+# activated experts of the captured cell (see profiles/): bytes per activated expert.  None
+# until an ncu capture has been summarised.
+NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 = None
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"], bf16_tflops_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def bits16(t):
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def make_cells(device):
+    w = WORKLOAD
+    cells = []
+    for a in w["alphas"]:
+        for s in w["seeds"]:
+            seed = 1000 * s + int(round(a * 100))
+            ids, wts, _ = di.routing_batch(seed, w["T"], w["k"], w["E"], a)
+            hist = np.bincount(ids.reshape(-1), minlength=w["E"])
+            cell = dict(alpha=a, seed=seed, ids=ids, w=wts, active=int((hist > 0).sum()), hist=hist)
+            if device is not None:
+                cell["x_host"] = di.activations(seed, w["T"], w["H"]).pin_memory()
+                cell["ids_host"] = torch.from_numpy(ids).pin_memory()
+                cell["w_host"] = torch.from_numpy(wts).pin_memory()
+                cell["x"] = cell["x_host"].to(device)
+                cell["ids_d"] = cell["ids_host"].to(device)
+                cell["w_d"] = cell["w_host"].to(device)
+            cells.append(cell)
+    return cells
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.perf_counter(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for t, r in self.rows if t0 <= t <= t1 + 0.11] or [r for _, r in self.rows]
+        sm, mx, reasons = [], [], set()
+        for r in rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def layer_bytes_flops(cell, tile_n):
+    """Algorithmic bytes and padded flops of one whole layer call (bf16)."""
+    w = WORKLOAD
+    P = w["T"] * w["k"]
+    A = cell["active"]
+    wbytes = A * 3 * w["H"] * w["I"] * 2
+    act = P * w["H"] * 2 * 2 + P * w["I"] * 2 * 2 + P * w["H"] * 4 * 2 + w["T"] * w["H"] * 2 * 2 + 16 * P
+    padded_cols = int(sum(-(-int(t) // tile_n) * tile_n for t in cell["hist"]))
+    return wbytes + act, padded_cols * 6 * w["H"] * w["I"], P * 6 * w["H"] * w["I"]
+
+
+def w13_launch_bytes(cell):
+    """Algorithmic bytes of one gate/up GEMM launch: each activated expert's W13 once, the
+    gathered activations read once, h written once."""
+    w = WORKLOAD
+    P = w["T"] * w["k"]
+    return cell["active"] * 2 * w["I"] * w["H"] * 2 + P * w["H"] * 2 + P * w["I"] * 2
+
+
+def oracle_sample_seconds(cells, n_tokens):
+    """Times the CPU oracle, as it stands, on the first n_tokens tokens of the first cell
+    (input generation excluded).  Returns (seconds, pairs in the sample)."""
+    from oracle import layer
+    w = WORKLOAD
+    W = di.MoEWeights(w["weight_seed"], w["E"], w["H"], w["I"])
+    cell = cells[0]
+    tokens = list(range(n_tokens))
+    need = sorted(set(int(e) for e in cell["ids"][tokens].reshape(-1)))
+    c13 = {e: bits16(W.expert_w13(e)) for e in need}
+    c2 = {e: bits16(W.expert_w2(e)) for e in need}
+    x = bits16(di.activations(cell["seed"], w["T"], w["H"]))
+    t0 = time.perf_counter()
+    layer.moe_layer_bf16(x, lambda e: c13[e], lambda e: c2[e], cell["ids"], cell["w"], w["E"], tokens=tokens)
+    return time.perf_counter() - t0, n_tokens * w["k"]
+
+
+def run_reference(args):
+    """The oracle timed on the host cores.  Each step is one (token, slot) pair of the workload
+    (the other slots of that token are masked with the skipped-id convention), scaled by the
+    512 pairs of a whole layer; the four experts it touches are generated once, outside the
+    timed region."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import layer
+    w = WORKLOAD
+    cell = make_cells(None)[0]
+    steps = args.steps if args.steps is not None else 8
+    warmup = args.warmup if args.warmup is not None else 1
+    P = w["T"] * w["k"]
+    W = di.MoEWeights(w["weight_seed"], w["E"], w["H"], w["I"])
+    x = bits16(di.activations(cell["seed"], w["T"], w["H"]))
+    n_pairs = 4
+    experts = [int(cell["ids"][0, j]) for j in range(n_pairs)]
+    c13 = {e: bits16(W.expert_w13(e)) for e in experts}
+    c2 = {e: bits16(W.expert_w2(e)) for e in experts}
+    times = []
+    for i in range(warmup + steps):
+        ids = np.full_like(cell["ids"], -1)
+        ids[0, i % n_pairs] = cell["ids"][0, i % n_pairs]
+        t0 = time.perf_counter()
+        layer.moe_layer_bf16(x, lambda e: c13[e], lambda e: c2[e], ids, cell["w"], w["E"], tokens=[0])
+        if i >= warmup:
+            times.append((time.perf_counter() - t0) * P)
+    us = statistics.mean(times) * 1e6
+    line = dict(metric="fused_moe_layer_us", value=us, unit="us", n_gpus=args.gpus, steps=steps, warmup=warmup,
+                ms_per_step=us / 1e3, higher_is_better=False, scaling="weak", vs_baseline=None, dtype="f64",
+                data="synthetic", impl="reference",
+                config=dict(workload=w["name"], E=w["E"], k=w["k"], H=w["H"], I=w["I"], T=w["T"]),
+                cpu_baseline=dict(value=us, unit="us", cores=torch.get_num_threads(), kind="oracle",
+                                  sample=f"one (token, slot) pair of {P} per step, scaled by {P} to a whole layer"),
+                e2e=dict(value=us, unit="us", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import paper_2607_23099_b200 as d
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    device = torch.device(f"cuda:{local}")
+    steps = args.steps if args.steps is not None else 320
+    warmup = args.warmup if args.warmup is not None else 16
+    warmup = max(3, warmup)
+    w = WORKLOAD
+    pk = peaks()
+
+    W = di.MoEWeights(w["weight_seed"], w["E"], w["H"], w["I"])
+    w13, w2 = W.materialize(device)
+    cells = make_cells(device)
+    m = d.DAMoE(w["T"], w["k"], w["E"], w["H"], w["I"], device=local)
+    table = "built-in cost model"
+    if os.path.exists(TABLE_PATH) and args.workload == "headline":
+        m.load_tuning_table(open(TABLE_PATH, "rb").read())
+        table = os.path.relpath(TABLE_PATH, ROOT)
+    out = torch.empty(w["T"], w["H"], dtype=torch.bfloat16, device=device)
+    stream = torch.cuda.current_stream()
+
+    def step(i, variant=d.VARIANT_AUTO):
+        c = cells[i % len(cells)]
+        m.fused_moe(c["x"], w13, w2, c["ids_d"], c["w_d"], variant, out=out, stream=stream)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+
+    # ---- timed region: K steps, device-timed, stage events on for the roofline figure ----
+    m.set_profiling(True)
+    sampler = ClockSampler(local)
+    time.sleep(0.25)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for i in range(steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop(t0, t1)
+    stage = m.stage_ms()
+    m.set_profiling(False)
+    status = m.debug_fetch(w["T"])["status"]
+
+    # ---- end to end through the host-buffer entry point ----
+    out_host = torch.empty(w["T"], w["H"], dtype=torch.bfloat16).pin_memory()
+    for i in range(3):
+        c = cells[i % len(cells)]
+        m.fused_moe_host(c["x_host"], w13, w2, c["ids_host"], c["w_host"], d.VARIANT_AUTO, out_host=out_host, stream=stream)
+    barrier()
+    torch.cuda.synchronize()
+    te0 = time.perf_counter()
+    for i in range(steps):
+        c = cells[i % len(cells)]
+        m.fused_moe_host(c["x_host"], w13, w2, c["ids_host"], c["w_host"], d.VARIANT_AUTO, out_host=out_host, stream=stream)
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - te0) * 1e3
+    barrier()
+
+    if world > 1:
+        t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=device)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms_total, e2e_ms = t.tolist()
+    us_per_layer = ms_total * 1e3 / steps
+    e2e_us = e2e_ms * 1e3 / steps
+
+    # ---- dispatch comparison per cell: AUTO vs STATIC vs every variant (median of 5) ----
+    def time_variant(ci, variant, reps=5):
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            step(ci, variant)
+            b.record(stream)
+            b.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3)
+        return statistics.median(ts)
+
+    ns = d.tile_ns()
+    per_cell = []
+    for ci, c in enumerate(cells):
+        t_auto = time_variant(ci, d.VARIANT_AUTO)
+        chosen = m.debug_fetch(w["T"])["variant_id"]
+        t_static = time_variant(ci, d.VARIANT_STATIC)
+        t_var = [time_variant(ci, v) for v in range(len(ns))]
+        nbytes, fl_pad, fl_use = layer_bytes_flops(c, ns[chosen])
+        t_roof = max(nbytes / (pk["hbm_gbs"] * 1e9), fl_pad / (pk["bf16_tflops_sustained"] * 1e12)) * 1e6
+        per_cell.append(dict(alpha=c["alpha"], seed=c["seed"], active=c["active"], auto_us=round(t_auto, 1),
+                             static_us=round(t_static, 1), best_us=round(min(t_var), 1), best_variant=int(np.argmin(t_var)),
+                             chosen=chosen, roofline_us=round(t_roof, 1), roofline_frac=round(t_roof / t_auto, 4),
+                             gbs=round(nbytes / t_auto / 1e3, 1), useful_tflops=round(fl_use / t_auto / 1e6, 2),
+                             padded_tflops=round(fl_pad / t_auto / 1e6, 2)))
+    geo = lambda xs: math.exp(sum(math.log(x) for x in xs) / len(xs))
+    dispatch = dict(geomean_speedup_vs_static=round(geo([c["static_us"] / c["auto_us"] for c in per_cell]), 4),
+                    geomean_gap_to_best=round(geo([c["auto_us"] / c["best_us"] for c in per_cell]), 4),
+                    layer_roofline_frac_mean=round(statistics.mean(c["roofline_frac"] for c in per_cell), 4),
+                    table=table, cells=per_cell)
+
+    if rank != 0:
+        return
+
+    # ---- roofline of the dominant kernel (gate/up grouped GEMM), from the timed region ----
+    n_rec = stage["calls"]
+    rec_cells = [cells[i % len(cells)] for i in range(steps - n_rec, steps)]
+    w13_bytes = statistics.mean(w13_launch_bytes(c) for c in rec_cells)
+    w13_ms = stage["gemm13"] / max(1, n_rec)
+    achieved = w13_bytes / (w13_ms * 1e-3) / 1e9
+    traffic = None
+    if NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 is not None:
+        traffic = NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 * statistics.mean(c["active"] for c in rec_cells)
+    roofline = dict(bound="hbm", kernel="gemm_branch_kernel<0> (grouped gate/up GEMM + SwiGLU)", achieved=round(achieved, 1),
+                    peak=pk["hbm_gbs"], unit="GB/s", frac=round(achieved / pk["hbm_gbs"], 4), traffic=traffic,
+                    peak_source=pk["source"], launch_ms=round(w13_ms, 4), launches_timed=n_rec,
+                    stage_share={k: round(stage[k] / max(1e-9, sum(stage[s] for s in m.STAGES)), 4) for k in m.STAGES})
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        sec, pairs = oracle_sample_seconds(cells, min(16, w["T"]))
+        P = w["T"] * w["k"]
+        cpu = dict(value=round(sec * P / pairs * 1e6, 1), unit="us", cores=torch.get_num_threads(), kind="oracle",
+                   sample=f"first {pairs // w['k']} of {w['T']} tokens ({pairs} of {P} pairs) of the first cell: {sec:.2f} s, scaled by {P // pairs}")
+
+    h2d = w["T"] * w["H"] * 2 + 2 * w["T"] * w["k"] * 4
+    d2h = w["T"] * w["H"] * 2
+    line = dict(metric="fused_moe_layer_us", value=round(us_per_layer, 2), unit="us", n_gpus=world, steps=steps,
+                warmup=warmup, ms_per_step=round(us_per_layer / 1e3, 5), higher_is_better=False, scaling="weak",
+                vs_baseline=None, dtype="bf16", data="synthetic",
+                config=dict(workload=w["name"], E=w["E"], k=w["k"], H=w["H"], I=w["I"], T=w["T"],
+                            alphas=w["alphas"], seeds_per_alpha=len(w["seeds"]), dispatch="auto/branch",
+                            l2="inputs larger than L2: every step streams 4-19 GB of expert weights",
+                            parallelism="replicas only" if world > 1 else "single GPU"),
+                aggregate_layers_per_s=round(world * 1e6 / us_per_layer, 2),
+                e2e=dict(value=round(e2e_us, 2), unit="us", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
+                gpu_launches=7 * steps, clocks=clocks, roofline=roofline, cpu_baseline=cpu, dispatch=dispatch,
+                device_status=status)
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="headline", choices=["headline", "small"],
+                    help="'small' is the reduced case used for ncu captures")
+    args = ap.parse_args()
+    if args.workload == "small":
+        WORKLOAD.clear()
+        WORKLOAD.update(SMALL_WORKLOAD)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

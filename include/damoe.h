@@ -164,6 +164,17 @@ int damoe_debug_fetch(damoe_ctx* ctx, int32_t* offsets, int32_t* perm, int32_t* 
                       int32_t* tiles, int32_t* variant_id, uint32_t* status_bits);
 
 /*
+ * Stage timing (diagnostic).  When enabled, damoe_fused_moe records CUDA events on the
+ * caller's stream around its five stages: route metadata + selection, token gather, gate/up
+ * GEMM, down GEMM, unpermute-reduce.  Up to 128 calls are remembered.
+ * damoe_get_stage_ms waits for the last recorded call, then writes the per-stage milliseconds
+ * summed over the remembered calls to ms[5], their number to *calls, and forgets them.
+ * Disabled by default; costs six event records per call when enabled.
+ */
+int damoe_set_profiling(damoe_ctx* ctx, int enabled);
+int damoe_get_stage_ms(damoe_ctx* ctx, float* ms, int* calls);
+
+/*
  * Dispatch microbenchmark (paper Section V-C, Table III): a producer kernel computes a value
  * that selects one of two trivial follow-up kernels.  Times `iters` repetitions of each of
  * three paths and writes the mean microseconds per repetition: us[0] copy the value to the

@@ -26,13 +26,14 @@ EXPORTS = [
     "damoe_create", "damoe_destroy", "damoe_last_error", "damoe_route_stats", "damoe_fused_moe",
     "damoe_fused_moe_host", "damoe_set_fp8_scales", "damoe_load_tuning_table", "damoe_set_dispatch",
     "damoe_variant_count", "damoe_variant_info", "damoe_debug_fetch", "damoe_dispatch_microbench",
+    "damoe_set_profiling", "damoe_get_stage_ms",
 ]
 
 
 def _load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
         raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2607_23099_b200.build` "
+            f"{LIB_PATH} is missing: build it with `python paper_2607_23099_b200/build.py` "
             "(needs nvcc with sm_100a support); there is no fallback path")
     lib = ctypes.CDLL(LIB_PATH)
     vp, i32, cp = ctypes.c_void_p, ctypes.c_int, ctypes.c_char_p
@@ -50,6 +51,8 @@ def _load() -> ctypes.CDLL:
     lib.damoe_variant_info.argtypes = [i32] + [ctypes.POINTER(i32)] * 4
     lib.damoe_debug_fetch.argtypes = [vp] * 7
     lib.damoe_dispatch_microbench.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_float)]
+    lib.damoe_set_profiling.argtypes = [vp, i32]
+    lib.damoe_get_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     for name in EXPORTS:
         if name != "damoe_last_error":
             getattr(lib, name).restype = i32
@@ -155,6 +158,18 @@ class DAMoE:
 
     def set_dispatch(self, mode: int):
         self._check(_lib.damoe_set_dispatch(self._ctx, mode))
+
+    STAGES = ("route", "gather", "gemm13", "gemm2", "reduce")
+
+    def set_profiling(self, enabled: bool):
+        self._check(_lib.damoe_set_profiling(self._ctx, int(enabled)))
+
+    def stage_ms(self) -> dict:
+        """Per-stage milliseconds summed over the calls recorded since the last query."""
+        ms = (ctypes.c_float * 5)()
+        n = ctypes.c_int()
+        self._check(_lib.damoe_get_stage_ms(self._ctx, ms, ctypes.byref(n)))
+        return dict(calls=n.value, **{k: ms[i] for i, k in enumerate(self.STAGES)})
 
     def debug_fetch(self, T: int) -> dict:
         """Routing metadata of the last fused_moe call (synchronises)."""

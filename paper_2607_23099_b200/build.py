@@ -1,4 +1,6 @@
-"""Builds libdamoe.so in-tree with nvcc for sm_100a.  `python -m paper_2607_23099_b200.build`"""
+"""Builds libdamoe.so in-tree with nvcc for sm_100a.  Run it as a script:
+`python paper_2607_23099_b200/build.py [--force] [-v]` (running it as a module would import the
+package first, which refuses to load without an up-to-date library)."""
 from __future__ import annotations
 
 import os

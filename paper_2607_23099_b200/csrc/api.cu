@@ -37,6 +37,10 @@ struct damoe_ctx {
   const void* cached_w2 = nullptr;
   // staging for the host-buffer entry point
   void *st_x = nullptr, *st_ids = nullptr, *st_w = nullptr, *st_out = nullptr;
+  // stage timing
+  bool profiling = false;
+  cudaEvent_t ev[128][6] = {};
+  int ev_count = 0;
   char err[256] = "";
 };
 
@@ -272,6 +276,9 @@ int damoe_create(damoe_ctx** out, int device, int max_T, int k, int E, int H, in
 int damoe_destroy(damoe_ctx* c) {
   if (!c) return DAMOE_OK;
   cudaSetDevice(c->device);
+  for (auto& set : c->ev)
+    for (auto& e : set)
+      if (e) cudaEventDestroy(e);
   if (c->arena) cudaFree(c->arena);
   if (c->table_blob) cudaFree(c->table_blob);
   delete c;
@@ -410,10 +417,22 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
   }
 
   c->last_T = T;
+  cudaEvent_t* ev = nullptr;
+  if (c->profiling) {
+    ev = c->ev[c->ev_count % 128];
+    for (int i = 0; i < 6; ++i)
+      if (!ev[i]) DAMOE_CUDA(c, cudaEventCreate(&ev[i]));
+    ++c->ev_count;
+  }
+#define DAMOE_MARK(i) \
+  if (ev) DAMOE_CUDA(c, cudaEventRecord(ev[i], st))
   SelectorArgs sel;
   const int known = make_selector(c, T, variant, &sel);
+  DAMOE_MARK(0);
   DAMOE_CUDA(c, launch_route(c->ws, topk_ids, topk_weights, T, c->k, c->E, sel, nullptr, nullptr, false, st));
+  DAMOE_MARK(1);
   DAMOE_CUDA(c, launch_gather(c->ws, static_cast<const __nv_bfloat16*>(x), T, c->k, c->H, st));
+  DAMOE_MARK(2);
 
   GemmMaps m13, m2;
   m13.w = c->map_w13;
@@ -434,15 +453,21 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
 
   if (known >= 0) {
     DAMOE_CUDA(c, launch_gemm(0, known, false, m13, ga, c->sm_count, st));
+    DAMOE_MARK(3);
     DAMOE_CUDA(c, launch_gemm(1, known, false, m2, ga, c->sm_count, st));
   } else if (c->dispatch == DAMOE_DISPATCH_PREDICATED) {
     for (int v = 0; v < kNumVariants; ++v) DAMOE_CUDA(c, launch_gemm(0, v, true, m13, ga, c->sm_count, st));
+    DAMOE_MARK(3);
     for (int v = 0; v < kNumVariants; ++v) DAMOE_CUDA(c, launch_gemm(1, v, true, m2, ga, c->sm_count, st));
   } else {
     DAMOE_CUDA(c, launch_gemm(0, -1, false, m13, ga, c->sm_count, st));
+    DAMOE_MARK(3);
     DAMOE_CUDA(c, launch_gemm(1, -1, false, m2, ga, c->sm_count, st));
   }
+  DAMOE_MARK(4);
   DAMOE_CUDA(c, launch_reduce(c->ws, static_cast<__nv_bfloat16*>(out), T, c->k, c->H, st));
+  DAMOE_MARK(5);
+#undef DAMOE_MARK
   return DAMOE_OK;
 }
 
@@ -464,6 +489,30 @@ int damoe_fused_moe_host(damoe_ctx* c, const void* x_host, const void* w13, cons
   if (rc != DAMOE_OK) return rc;
   DAMOE_CUDA(c, cudaMemcpyAsync(out_host, c->st_out, 2 * static_cast<size_t>(T) * c->H, cudaMemcpyDeviceToHost, st));
   DAMOE_CUDA(c, cudaStreamSynchronize(st));
+  return DAMOE_OK;
+}
+
+int damoe_set_profiling(damoe_ctx* c, int enabled) {
+  if (!c) return DAMOE_ERR_INVALID_ARG;
+  c->profiling = enabled != 0;
+  c->ev_count = 0;
+  return DAMOE_OK;
+}
+
+int damoe_get_stage_ms(damoe_ctx* c, float* ms, int* calls) {
+  if (!c || !ms) return DAMOE_ERR_INVALID_ARG;
+  DAMOE_CUDA(c, cudaSetDevice(c->device));
+  const int n = c->ev_count < 128 ? c->ev_count : 128;
+  for (int s = 0; s < 5; ++s) ms[s] = 0.f;
+  if (n > 0) DAMOE_CUDA(c, cudaEventSynchronize(c->ev[(c->ev_count - 1) % 128][5]));
+  for (int i = 0; i < n; ++i)
+    for (int s = 0; s < 5; ++s) {
+      float t = 0.f;
+      DAMOE_CUDA(c, cudaEventElapsedTime(&t, c->ev[i][s], c->ev[i][s + 1]));
+      ms[s] += t;
+    }
+  if (calls) *calls = n;
+  c->ev_count = 0;
   return DAMOE_OK;
 }
 

@@ -16,8 +16,8 @@ def _declared():
 
 @pytest.fixture(scope="module")
 def lib_path():
-    from paper_2607_23099_b200 import build
-    return build.build()
+    import __graft_entry__ as g
+    return g.load_build_module().build()
 
 
 def test_header_symbols_are_exported(lib_path):
