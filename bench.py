@@ -45,9 +45,10 @@ SMALL_WORKLOAD = dict(name="profile_small_E32_T8", E=32, k=8, H=7168, I=2048, T=
 TABLE_PATH = os.path.join(ROOT, "paper_2607_23099_b200", "tables", "e256_k8_h7168_i2048_bf16.damoetb")
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gate/up GEMM launch, divided by the
-# activated experts of the captured cell (see profiles/): bytes per activated expert.  None
-# until an ncu capture has been summarised.
-NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 = None
+# activated experts of the captured cell (profiles/gemm_gate_up_small_E32_T8_ncu_full.md):
+# bytes per activated expert.  The capture is of the reduced case; traffic grows in proportion
+# to the activated experts, so bench scales it by its own cells' counts.
+NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 = 59.05e6
 
 
 def peaks():
