@@ -98,6 +98,31 @@ int damoe_route_stats(damoe_ctx* ctx, const int32_t* topk_ids, int T, int k, int
                       int32_t* hist, double* eff_exp, void* stream);
 
 /*
+ * damoe_route_stats for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a convenience of this library.)  Some users of this code may not call
+ * cudaMalloc at all - an inference server that hands the whole GPU to its own memory pool at
+ * start-up has nothing left for cudaMalloc to give, and a latency-critical step loop cannot
+ * afford the device-wide synchronisation that cudaMalloc / cudaFree imply - and for them even
+ * damoe_create, which allocates the context's workspace, is off limits.  This entry point needs
+ * no context and allocates nothing, on the device or through any library: its scratch (the
+ * per-block partial histograms) is a fixed 512 KB array compiled into the library, which every
+ * GPU that loads the library keeps until the process exits.
+ *
+ * Same inputs, outputs and results as damoe_route_stats (hist dev [E] int32, eff_exp dev [1]
+ * double, bit-identical values), on the calling thread's current device.
+ * Limits: T * k <= 65536 pairs, else DAMOE_ERR_WORKSPACE; 1 <= k <= 32 and 1 <= E <= 1024,
+ * else DAMOE_ERR_UNSUPPORTED_SHAPE.
+ * The first call on each device looks up the scratch array's device address (one
+ * cudaGetSymbolAddress, no allocation); make that first call before any stream capture.
+ * All calls on a device share the one scratch array: calls whose kernels may overlap on the
+ * GPU (different streams without ordering) race with each other; serialise them.  The array
+ * keeps the previous call's contents; the call itself clears the one word that must start at
+ * zero, so the caller has nothing to reset.
+ */
+int damoe_route_stats_noalloc(const int32_t* topk_ids, int T, int k, int E, int32_t* hist,
+                              double* eff_exp, void* stream);
+
+/*
  * The whole layer (paper Section IV, Fig. 9(b) steps 5-6 plus the expert computation of
  * Section II-C): histogram and Effective Experts, stable grouping of (token, slot) pairs by
  * expert, per-variant padded-tile counts  tiles_v = sum_e ceil(t_e / N_v),  device-side choice

@@ -26,7 +26,7 @@ EXPORTS = [
     "damoe_create", "damoe_destroy", "damoe_last_error", "damoe_route_stats", "damoe_fused_moe",
     "damoe_fused_moe_host", "damoe_set_fp8_scales", "damoe_load_tuning_table", "damoe_set_dispatch",
     "damoe_variant_count", "damoe_variant_info", "damoe_debug_fetch", "damoe_dispatch_microbench",
-    "damoe_set_profiling", "damoe_get_stage_ms",
+    "damoe_set_profiling", "damoe_get_stage_ms", "damoe_route_stats_noalloc",
 ]
 
 
@@ -51,6 +51,7 @@ def _load() -> ctypes.CDLL:
     lib.damoe_variant_info.argtypes = [i32] + [ctypes.POINTER(i32)] * 4
     lib.damoe_debug_fetch.argtypes = [vp] * 7
     lib.damoe_dispatch_microbench.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_float)]
+    lib.damoe_route_stats_noalloc.argtypes = [vp, i32, i32, i32, vp, vp, vp]
     lib.damoe_set_profiling.argtypes = [vp, i32]
     lib.damoe_get_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     for name in EXPORTS:
@@ -94,6 +95,20 @@ def dispatch_microbench(iters: int = 200, device: int = 0) -> dict:
 
 def _ptr(t):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def route_stats_noalloc(topk_ids: torch.Tensor, E: int, hist: torch.Tensor, eff_exp: torch.Tensor, stream=None):
+    """Histogram and Effective Experts without a context and without any allocation: for
+    callers that may not call cudaMalloc (the GPU is fully owned by their own memory pool, or
+    the step loop cannot take cudaMalloc's device-wide synchronisation).  The caller passes
+    the outputs (hist [E] int32, eff_exp [1] float64, on the current CUDA device); scratch is a
+    fixed array inside the library, shared by all calls on that device, so overlapping calls
+    race.  At most 65536 (token, slot) pairs per call."""
+    T, k = topk_ids.shape
+    rc = _lib.damoe_route_stats_noalloc(_ptr(topk_ids), T, k, E, _ptr(hist), _ptr(eff_exp), _stream_ptr(stream))
+    if rc != OK:
+        raise DamoeError(rc, "damoe_route_stats_noalloc failed (size beyond the fixed scratch, bad shape or CUDA error)")
+    return hist, eff_exp
 
 
 def _stream_ptr(stream):

@@ -283,3 +283,67 @@ cudaError_t launch_route(const Workspace& ws, const int32_t* topk_ids, const flo
 }
 
 }  // namespace damoe
+
+// ---------------------------------------------------------------------------------------
+// Histogram + Effective Experts with no allocation anywhere: scratch lives in a file-scope
+// device array instead of a context's workspace.
+// ---------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kNoAllocMaxPairs = 65536;                                   // T * k accepted per call
+constexpr int kNoAllocMaxBlocks = kNoAllocMaxPairs / damoe::kPairsPerBlock;  // 128
+constexpr int kNoAllocWords = kNoAllocMaxBlocks * damoe::kMaxE + 64;      // per-block histograms + a status word
+
+// 512 KB + 256 B, resident on every GPU that loads the library until the process exits.
+// In host code this name is only a stand-in for the symbol; the device address comes from
+// cudaGetSymbolAddress below.
+static __device__ __align__(256) int32_t g_noalloc_scratch[kNoAllocWords];
+
+constexpr int kMaxDevices = 64;
+int32_t* g_noalloc_ptr[kMaxDevices] = {};
+
+// Once per device, with that device current: resolve the scratch array's device address.
+cudaError_t noalloc_scratch(int device, int32_t** out) {
+  if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!g_noalloc_ptr[device]) {
+    int32_t* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_noalloc_scratch);
+    if (e != cudaSuccess) return e;
+    g_noalloc_ptr[device] = p;
+  }
+  *out = g_noalloc_ptr[device];
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int damoe_route_stats_noalloc(const int32_t* topk_ids, int T, int k, int E, int32_t* hist, double* eff_exp,
+                                         void* stream) {
+  using namespace damoe;
+  if (!hist || !eff_exp || T < 0 || (T > 0 && !topk_ids)) return DAMOE_ERR_INVALID_ARG;
+  if (k < 1 || k > kMaxK || E < 1 || E > kMaxE) return DAMOE_ERR_UNSUPPORTED_SHAPE;
+  if (static_cast<long long>(T) * k > kNoAllocMaxPairs) return DAMOE_ERR_WORKSPACE;  // beyond the static scratch
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess) return DAMOE_ERR_CUDA;
+  int32_t* scratch = nullptr;
+  if (noalloc_scratch(device, &scratch) != cudaSuccess) return DAMOE_ERR_CUDA;
+  if (T == 0) {
+    if (cudaMemsetAsync(hist, 0, sizeof(int32_t) * E, st) != cudaSuccess) return DAMOE_ERR_CUDA;
+    if (cudaMemsetAsync(eff_exp, 0, sizeof(double), st) != cudaSuccess) return DAMOE_ERR_CUDA;
+    return DAMOE_OK;
+  }
+  // The per-block histograms are fully rewritten by the count kernel before the scan reads
+  // them; only the status word accumulates (atomicOr), so it alone is cleared here.
+  uint32_t* status = reinterpret_cast<uint32_t*>(scratch + kNoAllocMaxBlocks * kMaxE);
+  if (cudaMemsetAsync(status, 0, sizeof(uint32_t), st) != cudaSuccess) return DAMOE_ERR_CUDA;
+  Workspace ws{};
+  ws.block_hist = scratch;
+  ws.status = status;
+  SelectorArgs sel{};
+  const int P = T * k;
+  const int nblocks = (P + kPairsPerBlock - 1) / kPairsPerBlock;
+  route_count_kernel<<<nblocks, kPairsPerBlock, 0, st>>>(topk_ids, P, E, ws.block_hist, ws.status);
+  route_scan_kernel<<<1, kScanThreads, 0, st>>>(ws.block_hist, nblocks, E, ws, sel, hist, eff_exp, 1);
+  return cudaGetLastError() == cudaSuccess ? DAMOE_OK : DAMOE_ERR_CUDA;
+}

@@ -1,0 +1,56 @@
+"""The allocation-free histogram / Effective Experts entry point, for callers that may not call
+cudaMalloc (their own pool owns the whole GPU, or their step loop cannot take the device-wide
+synchronisation an allocation implies).  It must give exactly what the context-based entry
+point gives - integers and the binary64 statistic bit for bit - on two calls in a row, the
+second of which is smaller than the first so that anything left in the library's fixed
+scratch array by the first call would show.  Collected last on purpose."""
+import numpy as np
+import pytest
+import torch
+
+import damoe_inputs as di
+
+pytestmark = pytest.mark.gpu
+
+
+def _both(d, ctx, ids):
+    dev_ids = torch.from_numpy(ids).cuda()
+    E = ctx.E
+    want_hist, want_eff = ctx.route_stats(dev_ids)
+    hist = torch.full((E,), -7, dtype=torch.int32, device="cuda")
+    eff = torch.full((1,), -1.0, dtype=torch.float64, device="cuda")
+    d.route_stats_noalloc(dev_ids, E, hist, eff)
+    torch.cuda.synchronize()
+    return (hist.cpu().numpy(), eff.item()), (want_hist.cpu().numpy(), want_eff.item())
+
+
+def test_noalloc_matches_context_entry_point_twice_in_a_row():
+    import paper_2607_23099_b200 as d
+    E, k = 256, 8
+    ctx = d.DAMoE(8192, k, E, 1024, 512)
+    first, _, _ = di.routing_batch(21, 8192, k, E, 0.05)      # 65536 pairs: the entry point's maximum, 128 blocks
+    second, _, _ = di.routing_batch(22, 77, k, E, 10.0)       # 616 pairs: 2 blocks, ragged tail
+    second[3, 2] = -1                                         # a skipped id
+    for ids in (first, second):
+        got, want = _both(d, ctx, ids)
+        assert np.array_equal(got[0], want[0])
+        assert got[1] == want[1]
+        assert got[0].sum() == np.count_nonzero((ids >= 0) & (ids < E))
+    ctx.close()
+
+
+def test_noalloc_limits_and_empty_batch():
+    import paper_2607_23099_b200 as d
+    E, k = 64, 4
+    hist = torch.full((E,), 5, dtype=torch.int32, device="cuda")
+    eff = torch.full((1,), 5.0, dtype=torch.float64, device="cuda")
+    d.route_stats_noalloc(torch.empty(0, k, dtype=torch.int32, device="cuda"), E, hist, eff)
+    torch.cuda.synchronize()
+    assert hist.sum().item() == 0 and eff.item() == 0.0
+    too_big = torch.zeros(65536 // k + 1, k, dtype=torch.int32, device="cuda")
+    with pytest.raises(d.DamoeError) as ei:
+        d.route_stats_noalloc(too_big, E, hist, eff)
+    assert ei.value.code == 6
+    with pytest.raises(d.DamoeError) as ei:
+        d.route_stats_noalloc(too_big[:4], 2000, hist, eff)
+    assert ei.value.code == 2
