@@ -42,7 +42,18 @@ WORKLOAD = dict(name="deepseek_v3_decode_T64", E=256, k=8, H=7168, I=2048, T=64,
 # small; never the headline.
 SMALL_WORKLOAD = dict(name="profile_small_E32_T8", E=32, k=8, H=7168, I=2048, T=8,
                       alphas=[1.0], seeds=[0, 1], weight_seed=12345)
-TABLE_PATH = os.path.join(ROOT, "paper_2607_23099_b200", "tables", "e256_k8_h7168_i2048_bf16.damoetb")
+# Kimi-K2-shaped serving-trace stand-in: 500 batches, T log-uniform in [1, 4096], per-batch alpha
+# log-uniform in [0.05, 10]; adaptive vs static vs per-batch best variant.
+TRACE_WORKLOAD = dict(name="kimi_k2_trace_500", E=384, k=8, H=7168, I=2048, T=4096, trace=(1000, 500),
+                      weight_seed=12345)
+# The same kind of trace on the headline shape (weights already resident): 48 batches, part of
+# the default line so that the dispatcher is also measured where token counts and skew vary.
+HEADLINE_TRACE = (2000, 48)
+TABLE_DIR = os.path.join(ROOT, "paper_2607_23099_b200", "tables")
+
+
+def table_path(w):
+    return os.path.join(TABLE_DIR, f"e{w['E']}_k{w['k']}_h{w['H']}_i{w['I']}_bf16.damoetb")
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gate/up GEMM launch, divided by the
 # activated experts of the captured cell (profiles/gemm_gate_up_small_E32_T8_ncu_full.md):
@@ -64,17 +75,23 @@ def bits16(t):
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
-def make_cells(device):
+def make_cells(device, trace=None):
+    """The workload's batches.  trace = (seed, n) builds a serving-trace stand-in instead of
+    the fixed (alpha, seed) grid."""
     w = WORKLOAD
+    trace = trace if trace is not None else w.get("trace")
+    if trace is not None:
+        specs = [(T, a, trace[0] + i) for i, (T, a) in enumerate(di.trace_batches(trace[0], trace[1], t_max=w["T"]))]
+    else:
+        specs = [(w["T"], a, 1000 * s + int(round(a * 100))) for a in w["alphas"] for s in w["seeds"]]
     cells = []
-    for a in w["alphas"]:
-        for s in w["seeds"]:
-            seed = 1000 * s + int(round(a * 100))
-            ids, wts, _ = di.routing_batch(seed, w["T"], w["k"], w["E"], a)
+    for T, a, seed in specs:
+        if True:
+            ids, wts, _ = di.routing_batch(seed, T, w["k"], w["E"], a)
             hist = np.bincount(ids.reshape(-1), minlength=w["E"])
-            cell = dict(alpha=a, seed=seed, ids=ids, w=wts, active=int((hist > 0).sum()), hist=hist)
+            cell = dict(T=T, alpha=a, seed=seed, ids=ids, w=wts, active=int((hist > 0).sum()), hist=hist)
             if device is not None:
-                cell["x_host"] = di.activations(seed, w["T"], w["H"]).pin_memory()
+                cell["x_host"] = di.activations(seed, T, w["H"]).pin_memory()
                 cell["ids_host"] = torch.from_numpy(ids).pin_memory()
                 cell["w_host"] = torch.from_numpy(wts).pin_memory()
                 cell["x"] = cell["x_host"].to(device)
@@ -127,10 +144,10 @@ class ClockSampler:
 def layer_bytes_flops(cell, tile_n):
     """Algorithmic bytes and padded flops of one whole layer call (bf16)."""
     w = WORKLOAD
-    P = w["T"] * w["k"]
+    P = cell["T"] * w["k"]
     A = cell["active"]
     wbytes = A * 3 * w["H"] * w["I"] * 2
-    act = P * w["H"] * 2 * 2 + P * w["I"] * 2 * 2 + P * w["H"] * 4 * 2 + w["T"] * w["H"] * 2 * 2 + 16 * P
+    act = P * w["H"] * 2 * 2 + P * w["I"] * 2 * 2 + P * w["H"] * 4 * 2 + cell["T"] * w["H"] * 2 * 2 + 16 * P
     padded_cols = int(sum(-(-int(t) // tile_n) * tile_n for t in cell["hist"]))
     return wbytes + act, padded_cols * 6 * w["H"] * w["I"], P * 6 * w["H"] * w["I"]
 
@@ -139,7 +156,7 @@ def w13_launch_bytes(cell):
     """Algorithmic bytes of one gate/up GEMM launch: each activated expert's W13 once, the
     gathered activations read once, h written once."""
     w = WORKLOAD
-    P = w["T"] * w["k"]
+    P = cell["T"] * w["k"]
     return cell["active"] * 2 * w["I"] * w["H"] * 2 + P * w["H"] * 2 + P * w["I"] * 2
 
 
@@ -154,7 +171,7 @@ def oracle_sample_seconds(cells, n_tokens):
     need = sorted(set(int(e) for e in cell["ids"][tokens].reshape(-1)))
     c13 = {e: bits16(W.expert_w13(e)) for e in need}
     c2 = {e: bits16(W.expert_w2(e)) for e in need}
-    x = bits16(di.activations(cell["seed"], w["T"], w["H"]))
+    x = bits16(di.activations(cell["seed"], cell["T"], w["H"]))
     t0 = time.perf_counter()
     layer.moe_layer_bf16(x, lambda e: c13[e], lambda e: c2[e], cell["ids"], cell["w"], w["E"], tokens=tokens)
     return time.perf_counter() - t0, n_tokens * w["k"]
@@ -175,7 +192,7 @@ def run_reference(args):
     warmup = args.warmup if args.warmup is not None else 1
     P = w["T"] * w["k"]
     W = di.MoEWeights(w["weight_seed"], w["E"], w["H"], w["I"])
-    x = bits16(di.activations(cell["seed"], w["T"], w["H"]))
+    x = bits16(di.activations(cell["seed"], cell["T"], w["H"]))
     n_pairs = 4
     experts = [int(cell["ids"][0, j]) for j in range(n_pairs)]
     c13 = {e: bits16(W.expert_w13(e)) for e in experts}
@@ -199,6 +216,61 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def max_over_ranks(values, world, device=None):
+    """Element-wise MAX of a list of floats over all ranks (identity when world == 1)."""
+    if world <= 1:
+        return list(values)
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def geomean(xs):
+    xs = list(xs)
+    return math.exp(sum(math.log(x) for x in xs) / len(xs))
+
+
+def compare_dispatch(m, d, cells, run, pk, reps=3):
+    """Per batch: AUTO vs STATIC vs every variant (median of reps), roofline of the chosen one."""
+    ns = d.tile_ns()
+    stream = torch.cuda.current_stream()
+
+    def time_variant(c, variant):
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            run(c, variant)
+            b.record(stream)
+            b.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3)
+        return statistics.median(ts)
+
+    rows = []
+    for c in cells:
+        run(c, d.VARIANT_AUTO)
+        t_auto = time_variant(c, d.VARIANT_AUTO)
+        chosen = m.debug_fetch(c["T"])["variant_id"]
+        run(c, d.VARIANT_STATIC)
+        t_static = time_variant(c, d.VARIANT_STATIC)
+        static_id = m.debug_fetch(c["T"])["variant_id"]
+        t_var = [time_variant(c, v) for v in range(len(ns))]
+        nbytes, fl_pad, fl_use = layer_bytes_flops(c, ns[chosen])
+        t_roof = max(nbytes / (pk["hbm_gbs"] * 1e9), fl_pad / (pk["bf16_tflops_sustained"] * 1e12)) * 1e6
+        rows.append(dict(T=c["T"], alpha=round(c["alpha"], 4), active=c["active"], auto_us=round(t_auto, 1),
+                         static_us=round(t_static, 1), best_us=round(min(t_var), 1), best_variant=int(np.argmin(t_var)),
+                         chosen=chosen, static_variant=static_id, roofline_us=round(t_roof, 1),
+                         roofline_frac=round(t_roof / t_auto, 4), gbs=round(nbytes / t_auto / 1e3, 1),
+                         useful_tflops=round(fl_use / t_auto / 1e6, 2), padded_tflops=round(fl_pad / t_auto / 1e6, 2)))
+    ratios = [r["static_us"] / r["auto_us"] for r in rows]
+    return dict(geomean_speedup_vs_static=round(geomean(ratios), 4), peak_speedup_vs_static=round(max(ratios), 4),
+                geomean_gap_to_best=round(geomean(r["auto_us"] / r["best_us"] for r in rows), 4),
+                geomean_static_gap_to_best=round(geomean(r["static_us"] / r["best_us"] for r in rows), 4),
+                layer_roofline_frac_mean=round(statistics.mean(r["roofline_frac"] for r in rows), 4),
+                layer_roofline_frac_min=round(min(r["roofline_frac"] for r in rows), 4), batches=len(rows)), rows
+
+
 def run_ours(args):
     import paper_2607_23099_b200 as d
 
@@ -210,10 +282,10 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     torch.cuda.set_device(local)
     device = torch.device(f"cuda:{local}")
-    steps = args.steps if args.steps is not None else 320
-    warmup = args.warmup if args.warmup is not None else 16
-    warmup = max(3, warmup)
     w = WORKLOAD
+    is_trace = "trace" in w
+    steps = args.steps if args.steps is not None else (w["trace"][1] if is_trace else 320)
+    warmup = max(3, args.warmup if args.warmup is not None else 16)
     pk = peaks()
 
     W = di.MoEWeights(w["weight_seed"], w["E"], w["H"], w["I"])
@@ -221,22 +293,26 @@ def run_ours(args):
     cells = make_cells(device)
     m = d.DAMoE(w["T"], w["k"], w["E"], w["H"], w["I"], device=local)
     table = "built-in cost model"
-    if os.path.exists(TABLE_PATH) and args.workload == "headline":
-        m.load_tuning_table(open(TABLE_PATH, "rb").read())
-        table = os.path.relpath(TABLE_PATH, ROOT)
+    if os.path.exists(table_path(w)) and not args.no_table:
+        m.load_tuning_table(open(table_path(w), "rb").read())
+        table = os.path.relpath(table_path(w), ROOT)
     out = torch.empty(w["T"], w["H"], dtype=torch.bfloat16, device=device)
+    out_host = torch.empty(w["T"], w["H"], dtype=torch.bfloat16).pin_memory()
     stream = torch.cuda.current_stream()
 
-    def step(i, variant=d.VARIANT_AUTO):
-        c = cells[i % len(cells)]
-        m.fused_moe(c["x"], w13, w2, c["ids_d"], c["w_d"], variant, out=out, stream=stream)
+    def run(c, variant=d.VARIANT_AUTO):
+        m.fused_moe(c["x"], w13, w2, c["ids_d"], c["w_d"], variant, out=out[:c["T"]], stream=stream)
+
+    def run_host(c):
+        m.fused_moe_host(c["x_host"], w13, w2, c["ids_host"], c["w_host"], d.VARIANT_AUTO, out_host=out_host[:c["T"]],
+                         stream=stream)
 
     def barrier():
         if world > 1:
             torch.distributed.barrier()
 
     for i in range(warmup):
-        step(i)
+        run(cells[i % len(cells)])
     torch.cuda.synchronize()
 
     # ---- timed region: K steps, device-timed, stage events on for the roofline figure ----
@@ -249,7 +325,7 @@ def run_ours(args):
     t0 = time.perf_counter()
     e0.record(stream)
     for i in range(steps):
-        step(i)
+        run(cells[i % len(cells)])
     e1.record(stream)
     torch.cuda.synchronize()
     t1 = time.perf_counter()
@@ -258,61 +334,31 @@ def run_ours(args):
     clocks = sampler.stop(t0, t1)
     stage = m.stage_ms()
     m.set_profiling(False)
-    status = m.debug_fetch(w["T"])["status"]
+    status = m.debug_fetch(cells[(steps - 1) % len(cells)]["T"])["status"]
 
-    # ---- end to end through the host-buffer entry point ----
-    out_host = torch.empty(w["T"], w["H"], dtype=torch.bfloat16).pin_memory()
+    # ---- end to end through the host-buffer entry point (pinned host inputs and output) ----
     for i in range(3):
-        c = cells[i % len(cells)]
-        m.fused_moe_host(c["x_host"], w13, w2, c["ids_host"], c["w_host"], d.VARIANT_AUTO, out_host=out_host, stream=stream)
+        run_host(cells[i % len(cells)])
     barrier()
     torch.cuda.synchronize()
     te0 = time.perf_counter()
     for i in range(steps):
-        c = cells[i % len(cells)]
-        m.fused_moe_host(c["x_host"], w13, w2, c["ids_host"], c["w_host"], d.VARIANT_AUTO, out_host=out_host, stream=stream)
+        run_host(cells[i % len(cells)])
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - te0) * 1e3
     barrier()
 
-    if world > 1:
-        t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=device)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms_total, e2e_ms = t.tolist()
+    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms], world, device)
     us_per_layer = ms_total * 1e3 / steps
     e2e_us = e2e_ms * 1e3 / steps
 
-    # ---- dispatch comparison per cell: AUTO vs STATIC vs every variant (median of 5) ----
-    def time_variant(ci, variant, reps=5):
-        ts = []
-        for _ in range(reps):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            step(ci, variant)
-            b.record(stream)
-            b.synchronize()
-            ts.append(a.elapsed_time(b) * 1e3)
-        return statistics.median(ts)
-
-    ns = d.tile_ns()
-    per_cell = []
-    for ci, c in enumerate(cells):
-        t_auto = time_variant(ci, d.VARIANT_AUTO)
-        chosen = m.debug_fetch(w["T"])["variant_id"]
-        t_static = time_variant(ci, d.VARIANT_STATIC)
-        t_var = [time_variant(ci, v) for v in range(len(ns))]
-        nbytes, fl_pad, fl_use = layer_bytes_flops(c, ns[chosen])
-        t_roof = max(nbytes / (pk["hbm_gbs"] * 1e9), fl_pad / (pk["bf16_tflops_sustained"] * 1e12)) * 1e6
-        per_cell.append(dict(alpha=c["alpha"], seed=c["seed"], active=c["active"], auto_us=round(t_auto, 1),
-                             static_us=round(t_static, 1), best_us=round(min(t_var), 1), best_variant=int(np.argmin(t_var)),
-                             chosen=chosen, roofline_us=round(t_roof, 1), roofline_frac=round(t_roof / t_auto, 4),
-                             gbs=round(nbytes / t_auto / 1e3, 1), useful_tflops=round(fl_use / t_auto / 1e6, 2),
-                             padded_tflops=round(fl_pad / t_auto / 1e6, 2)))
-    geo = lambda xs: math.exp(sum(math.log(x) for x in xs) / len(xs))
-    dispatch = dict(geomean_speedup_vs_static=round(geo([c["static_us"] / c["auto_us"] for c in per_cell]), 4),
-                    geomean_gap_to_best=round(geo([c["auto_us"] / c["best_us"] for c in per_cell]), 4),
-                    layer_roofline_frac_mean=round(statistics.mean(c["roofline_frac"] for c in per_cell), 4),
-                    table=table, cells=per_cell)
+    # ---- adaptive vs static vs per-batch best ----
+    summary, rows = compare_dispatch(m, d, cells, run, pk)
+    dispatch = dict(summary, table=table, cells=rows if len(rows) <= 64 else rows[:64])
+    if not is_trace and args.workload == "headline":
+        tcells = make_cells(device, trace=HEADLINE_TRACE)
+        tsum, trows = compare_dispatch(m, d, tcells, run, pk)
+        dispatch["trace"] = dict(tsum, what="48 batches, T log-uniform [1, 64], alpha log-uniform [0.05, 10]")
 
     if rank != 0:
         return
@@ -323,30 +369,34 @@ def run_ours(args):
     w13_bytes = statistics.mean(w13_launch_bytes(c) for c in rec_cells)
     w13_ms = stage["gemm13"] / max(1, n_rec)
     achieved = w13_bytes / (w13_ms * 1e-3) / 1e9
-    traffic = None
-    if NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 is not None:
-        traffic = NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 * statistics.mean(c["active"] for c in rec_cells)
+    traffic = NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 * statistics.mean(c["active"] for c in rec_cells)
     roofline = dict(bound="hbm", kernel="gemm_branch_kernel<0> (grouped gate/up GEMM + SwiGLU)", achieved=round(achieved, 1),
-                    peak=pk["hbm_gbs"], unit="GB/s", frac=round(achieved / pk["hbm_gbs"], 4), traffic=traffic,
-                    peak_source=pk["source"], launch_ms=round(w13_ms, 4), launches_timed=n_rec,
+                    peak=pk["hbm_gbs"], unit="GB/s", frac=round(achieved / pk["hbm_gbs"], 4), traffic=round(traffic),
+                    algorithmic_bytes=round(w13_bytes), peak_source=pk["source"], launch_ms=round(w13_ms, 4),
+                    launches_timed=n_rec,
                     stage_share={k: round(stage[k] / max(1e-9, sum(stage[s] for s in m.STAGES)), 4) for k in m.STAGES})
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        sec, pairs = oracle_sample_seconds(cells, min(16, w["T"]))
-        P = w["T"] * w["k"]
+        n_tok = min(16, cells[0]["T"])
+        sec, pairs = oracle_sample_seconds(cells, n_tok)
+        P = cells[0]["T"] * w["k"]
         cpu = dict(value=round(sec * P / pairs * 1e6, 1), unit="us", cores=torch.get_num_threads(), kind="oracle",
-                   sample=f"first {pairs // w['k']} of {w['T']} tokens ({pairs} of {P} pairs) of the first cell: {sec:.2f} s, scaled by {P // pairs}")
+                   sample=f"first {n_tok} of {cells[0]['T']} tokens ({pairs} of {P} pairs) of the first batch: {sec:.2f} s, "
+                          f"scaled by {P / pairs:g}")
 
-    h2d = w["T"] * w["H"] * 2 + 2 * w["T"] * w["k"] * 4
-    d2h = w["T"] * w["H"] * 2
+    mean_T = statistics.mean(c["T"] for c in cells)
+    h2d = int(mean_T * w["H"] * 2 + 2 * mean_T * w["k"] * 4)
+    d2h = int(mean_T * w["H"] * 2)
+    config = dict(workload=w["name"], E=w["E"], k=w["k"], H=w["H"], I=w["I"], T=w["T"] if not is_trace else "log-uniform [1, 4096]",
+                  batches=len(cells), dispatch="auto/branch", table=table,
+                  l2="inputs larger than L2: a step streams the activated experts' weights (GBs), never reused across steps",
+                  parallelism="replicas only" if world > 1 else "single GPU")
+    if not is_trace:
+        config.update(alphas=w["alphas"], seeds_per_alpha=len(w["seeds"]))
     line = dict(metric="fused_moe_layer_us", value=round(us_per_layer, 2), unit="us", n_gpus=world, steps=steps,
                 warmup=warmup, ms_per_step=round(us_per_layer / 1e3, 5), higher_is_better=False, scaling="weak",
-                vs_baseline=None, dtype="bf16", data="synthetic",
-                config=dict(workload=w["name"], E=w["E"], k=w["k"], H=w["H"], I=w["I"], T=w["T"],
-                            alphas=w["alphas"], seeds_per_alpha=len(w["seeds"]), dispatch="auto/branch",
-                            l2="inputs larger than L2: every step streams 4-19 GB of expert weights",
-                            parallelism="replicas only" if world > 1 else "single GPU"),
+                vs_baseline=None, dtype="bf16", data="synthetic", config=config,
                 aggregate_layers_per_s=round(world * 1e6 / us_per_layer, 2),
                 e2e=dict(value=round(e2e_us, 2), unit="us", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
                 gpu_launches=7 * steps, clocks=clocks, roofline=roofline, cpu_baseline=cpu, dispatch=dispatch,
@@ -361,12 +411,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="headline", choices=["headline", "small"],
-                    help="'small' is the reduced case used for ncu captures")
+    ap.add_argument("--workload", default="headline", choices=["headline", "small", "kimi_trace"],
+                    help="'small' is the reduced case used for ncu captures; 'kimi_trace' the 500-batch serving-trace stand-in")
+    ap.add_argument("--no-table", action="store_true", help="ignore the committed tuning table")
     args = ap.parse_args()
-    if args.workload == "small":
+    if args.workload != "headline":
         WORKLOAD.clear()
-        WORKLOAD.update(SMALL_WORKLOAD)
+        WORKLOAD.update(SMALL_WORKLOAD if args.workload == "small" else TRACE_WORKLOAD)
     if args.impl == "reference":
         run_reference(args)
     else:

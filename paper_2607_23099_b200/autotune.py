@@ -1,0 +1,213 @@
+"""Offline auto-tuning (paper Section IV-A, Fig. 9(a)).
+
+For every token-count bucket: generate synthetic routings over a sweep of Dirichlet skews,
+time every kernel variant of the library on each, and record per distribution the exemplar
+(sorted, L2-normalised per-expert count vector; centroid over the samples, re-normalised) with
+the variant of lowest mean latency.  The static per-bucket entry - the baseline the paper calls
+NoDA - is the best variant under uniform random routing.  Besides the exemplar table the sweep
+also fits the coefficients of the integer cost model and Effective-Experts bins.
+
+    python -m paper_2607_23099_b200.autotune --shape dsv3 [--buckets 1,4,...] [--alphas ...]
+        [--seeds 3] [--reps 3] [--mode exemplar|bins|cost] --out table.damoetb [--log sweep.jsonl]
+
+The sweep log is append-only JSON lines, one per (T, alpha, seed, variant) timing, and a rerun
+skips what the log already holds, so an interrupted sweep resumes.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import damoe_inputs as di  # noqa: E402
+import paper_2607_23099_b200 as d  # noqa: E402
+from paper_2607_23099_b200 import tuning  # noqa: E402
+
+SHAPES = {
+    "tiny": dict(E=8, k=2, H=1024, I=512),
+    "dsv3": dict(E=256, k=8, H=7168, I=2048),
+    "kimi": dict(E=384, k=8, H=7168, I=2048),
+}
+UNIFORM = "uniform"
+
+
+# ---- host-side table content (pure numpy; no GPU needed) -----------------------------
+
+def sorted_unit(counts) -> np.ndarray:
+    q = np.sort(np.asarray(counts, dtype=np.float64))[::-1]
+    n = math.sqrt(float(np.dot(q, q)))
+    return q / n if n > 0 else q
+
+
+def exemplar_q30(count_vectors) -> list:
+    """Centroid of the samples' sorted unit vectors, re-normalised, as round(e * 2^30)."""
+    c = np.mean([sorted_unit(v) for v in count_vectors], axis=0)
+    n = math.sqrt(float(np.dot(c, c)))
+    if n > 0:
+        c = c / n
+    return [int(v) for v in np.rint(c * float(1 << 30))]
+
+
+def effective_experts(counts) -> float:
+    c = np.asarray(counts, dtype=np.float64)
+    s2 = float(np.dot(c, c))
+    return float(c.sum()) ** 2 / s2 if s2 > 0 else 0.0
+
+
+def fit_cost(rows, ns):
+    """Least-squares fit, per variant, of t = c_fix + c_byte*A + c_reload*(tiles - A) on the
+    cells where the memory term dominates and of c_flop on the others; picoseconds, >= 0."""
+    V = len(ns)
+    out = dict(c_fix=[0] * V, c_byte=[0] * V, c_reload=[0] * V, c_flop=[0] * V)
+    for v in range(V):
+        pts = [(r["active"], r["tiles"][v], r["us"][v]) for r in rows]
+        if not pts:
+            continue
+        A = np.array([[1.0, a, max(0, t - a)] for a, t, _ in pts])
+        y = np.array([us * 1e6 for _, _, us in pts])
+        coef, *_ = np.linalg.lstsq(A, y, rcond=None)
+        coef = np.maximum(coef, 0.0)
+        out["c_fix"][v], out["c_byte"][v], out["c_reload"][v] = (int(min(c, 2 ** 35)) for c in coef)
+        # compute floor: the fastest observed time per padded column bounds c_flop from above
+        per_col = min(us * 1e6 / max(1, t * ns[v]) for _, t, us in pts)
+        out["c_flop"][v] = int(min(per_col, 2 ** 35))
+    return out
+
+
+def build_bucket(T, cells, ns, V):
+    """cells: list of dict(alpha, counts[S][E], us[S][V], active[S], tiles[S][V])."""
+    ex, exv, rows, effs = [], [], [], []
+    static_variant = 2
+    for c in cells:
+        mean_us = np.mean(np.array(c["us"]), axis=0)
+        best = int(np.argmin(mean_us))
+        if c["alpha"] == UNIFORM:
+            static_variant = best
+        else:
+            ex.append(exemplar_q30(c["counts"]))
+            exv.append(best)
+            effs.append((float(np.mean([effective_experts(h) for h in c["counts"]])), best))
+        for s in range(len(c["us"])):
+            rows.append(dict(active=c["active"][s], tiles=c["tiles"][s], us=c["us"][s]))
+    # Effective-Experts bins: thresholds halfway between neighbouring distributions whose best variant differs
+    effs.sort()
+    thr, binv = [], []
+    for (e0, v0), (e1, v1) in zip(effs, effs[1:]):
+        if v0 != v1:
+            thr.append(int((e0 + e1) / 2 * 65536))
+            binv.append(v0)
+    binv.append(effs[-1][1] if effs else static_variant)
+    b = dict(T=T, static_variant=static_variant, exemplars=ex, exemplar_variants=exv, bin_thresholds_num=thr,
+             bin_den=65536, bin_variants=binv)
+    b.update(fit_cost(rows, ns))
+    return b
+
+
+# ---- the sweep (GPU) ---------------------------------------------------------------------
+
+def time_call(fn, reps):
+    ts = []
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        b.synchronize()
+        ts.append(a.elapsed_time(b) * 1e3)
+    return statistics.median(ts)
+
+
+def sweep(shape, buckets, alphas, seeds, reps, log_path, weight_seed=12345, device="cuda:0"):
+    E, k, H, I = shape["E"], shape["k"], shape["H"], shape["I"]
+    V, ns = d.variant_count(), d.tile_ns()
+    done = {}
+    if log_path and os.path.exists(log_path):
+        for line in open(log_path):
+            r = json.loads(line)
+            done[(r["T"], str(r["alpha"]), r["seed"])] = r
+    W = di.MoEWeights(weight_seed, E, H, I)
+    w13, w2 = W.materialize(device)
+    m = d.DAMoE(max(buckets), k, E, H, I)
+    log = open(log_path, "a") if log_path else None
+    result = {}
+    for T in buckets:
+        cells = []
+        for alpha in list(alphas) + [UNIFORM]:
+            cell = dict(alpha=alpha, counts=[], us=[], active=[], tiles=[])
+            for s in range(seeds):
+                key = (T, str(alpha), s)
+                if key in done:
+                    r = done[key]
+                else:
+                    seed = 50000 + 977 * s + T            # tuning seeds, disjoint from evaluation seeds
+                    if alpha == UNIFORM:
+                        ids, wts = di.uniform_routing(seed, T, k, E)
+                    else:
+                        ids, wts, _ = di.routing_batch(seed + int(round(alpha * 1000)), T, k, E, alpha)
+                    x = di.activations(seed, T, H, device)
+                    ids_d, w_d = torch.from_numpy(ids).to(device), torch.from_numpy(wts).to(device)
+                    out = torch.empty(T, H, dtype=torch.bfloat16, device=device)
+                    for v in range(V):                       # warm-up
+                        m.fused_moe(x, w13, w2, ids_d, w_d, v, out=out)
+                    us = [time_call(lambda v=v: m.fused_moe(x, w13, w2, ids_d, w_d, v, out=out), reps) for v in range(V)]
+                    meta = m.debug_fetch(T)
+                    hist = np.bincount(ids.reshape(-1), minlength=E)
+                    r = dict(T=T, alpha=alpha, seed=s, us=us, counts=hist.tolist(), active=int((hist > 0).sum()),
+                             tiles=meta["tiles"].tolist(), status=meta["status"])
+                    if log:
+                        log.write(json.dumps(r) + "\n")
+                        log.flush()
+                cell["counts"].append(r["counts"])
+                cell["us"].append(r["us"])
+                cell["active"].append(r["active"])
+                cell["tiles"].append(r["tiles"])
+            cells.append(cell)
+        result[T] = cells
+    m.close()
+    return result, ns, V
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--shape", default="dsv3", choices=sorted(SHAPES))
+    ap.add_argument("--buckets", default="1,4,16,64,256,1024,4096,8192")
+    ap.add_argument("--alphas", default="0.05,0.2,1,10")
+    ap.add_argument("--seeds", type=int, default=3)
+    ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--mode", default="exemplar", choices=["exemplar", "bins", "cost"])
+    ap.add_argument("--out", required=True)
+    ap.add_argument("--log", default=None)
+    args = ap.parse_args()
+    shape = SHAPES[args.shape]
+    buckets = [int(t) for t in args.buckets.split(",")]
+    alphas = [float(a) for a in args.alphas.split(",")]
+    result, ns, V = sweep(shape, buckets, alphas, args.seeds, args.reps, args.log)
+    table = dict(mode=dict(exemplar=d.MODE_EXEMPLAR, bins=d.MODE_EFFEXP_BINS, cost=d.MODE_COST)[args.mode],
+                 buckets=[build_bucket(T, result[T], ns, V) for T in buckets])
+    blob = tuning.pack_table(table, shape["E"], shape["k"], shape["H"], shape["I"], d.BF16, V)
+    os.makedirs(os.path.dirname(os.path.abspath(args.out)), exist_ok=True)
+    open(args.out, "wb").write(blob)
+    # landscape report
+    print(f"# variants N = {ns}; microseconds per layer, mean over {args.seeds} seeds; * = best")
+    for T in buckets:
+        for c in result[T]:
+            mean_us = np.mean(np.array(c["us"]), axis=0)
+            best = int(np.argmin(mean_us))
+            eff = np.mean([effective_experts(h) for h in c["counts"]])
+            cols = " ".join(f"{u:9.1f}{'*' if v == best else ' '}" for v, u in enumerate(mean_us))
+            print(f"T={T:5d} alpha={str(c['alpha']):>7s} eff={eff:6.1f} A={np.mean(c['active']):6.1f} | {cols}")
+    print(f"wrote {args.out} ({len(blob)} bytes)")
+
+
+if __name__ == "__main__":
+    main()
