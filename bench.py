@@ -148,7 +148,8 @@ def layer_bytes_flops(cell, tile_n):
     A = cell["active"]
     wbytes = A * 3 * w["H"] * w["I"] * 2
     act = P * w["H"] * 2 * 2 + P * w["I"] * 2 * 2 + P * w["H"] * 4 * 2 + cell["T"] * w["H"] * 2 * 2 + 16 * P
-    padded_cols = int(sum(-(-int(t) // tile_n) * tile_n for t in cell["hist"]))
+    # full tiles cost tile_n columns; the ragged last tile of an expert issues MMAs of ceil16(rest) columns
+    padded_cols = int(sum((int(t) // tile_n) * tile_n + (-(-(int(t) % tile_n) // 16) * 16) for t in cell["hist"]))
     return wbytes + act, padded_cols * 6 * w["H"] * w["I"], P * 6 * w["H"] * w["I"]
 
 

@@ -125,6 +125,18 @@ class MoEWeights:
         n = self.H * self.I
         return normal_bf16(self.seed, TID_W2, e * n, n, self.sigma, device).view(self.H, self.I)
 
+    def materialize_fp8(self, device):
+        """(w13q, w13_scale, w2q, w2_scale): E4M3 codes with 128x128 block scales."""
+        E, H, I = self.E, self.H, self.I
+        w13q = torch.empty(E, 2 * I, H, dtype=torch.uint8, device=device)
+        w2q = torch.empty(E, H, I, dtype=torch.uint8, device=device)
+        w13s = torch.empty(E, 2 * I // 128, H // 128, dtype=torch.float32, device=device)
+        w2s = torch.empty(E, H // 128, I // 128, dtype=torch.float32, device=device)
+        for e in range(E):
+            w13q[e], w13s[e] = quantize_e4m3_blocks(self.expert_w13(e, device), 128, 128)
+            w2q[e], w2s[e] = quantize_e4m3_blocks(self.expert_w2(e, device), 128, 128)
+        return w13q, w13s, w2q, w2s
+
     def materialize(self, device):
         w13 = torch.empty(self.E, 2 * self.I, self.H, dtype=torch.bfloat16, device=device)
         w2 = torch.empty(self.E, self.H, self.I, dtype=torch.bfloat16, device=device)
@@ -132,6 +144,19 @@ class MoEWeights:
             w13[e] = self.expert_w13(e, device)
             w2[e] = self.expert_w2(e, device)
         return w13, w2
+
+
+def quantize_e4m3_blocks(t: torch.Tensor, block_rows: int, block_cols: int):
+    """Block-scaled FP8 form of a bf16 matrix [R, C]: one fp32 scale per block_rows x block_cols
+    block, scale = amax / 448 (1 for an all-zero block), codes = e4m3(value / scale) as uint8.
+    Returns (codes [R, C] uint8, scales [R/block_rows, C/block_cols] float32).  This only
+    prepares inputs for the FP8 configuration; it is not part of the measured path."""
+    R, C = t.shape
+    v = t.float().view(R // block_rows, block_rows, C // block_cols, block_cols)
+    amax = v.abs().amax(dim=(1, 3))
+    scale = torch.where(amax == 0, torch.ones_like(amax), amax / 448.0)
+    q = (v / scale[:, None, :, None]).clamp(-448.0, 448.0).to(torch.float8_e4m3fn)
+    return q.view(torch.uint8).view(R, C), scale
 
 
 def activations(seed: int, T: int, H: int, device="cpu") -> torch.Tensor:

@@ -77,8 +77,16 @@ enum { DAMOE_MODE_EXEMPLAR = 0, DAMOE_MODE_EFFEXP_BINS = 1, DAMOE_MODE_COST = 2 
  * metadata, the permuted activations [max_T*k, H] bf16, the intermediate h [max_T*k, I] bf16
  * and the per-pair down-projection results [max_T*k, H] fp32.  `device` becomes the current
  * device of the calling thread.  Requirements: 1 <= k <= 32, 1 <= E <= 1024, H and I
- * multiples of 128.  dtype DAMOE_FP8_E4M3_BLOCK128 is declared but not implemented yet:
- * damoe_create returns DAMOE_ERR_UNSUPPORTED_SHAPE for it.
+ * multiples of 128, max_T * k <= 131072.
+ *
+ * dtype DAMOE_FP8_E4M3_BLOCK128: x, w13, w2 hold one-byte E4M3 codes (same shapes) with fp32
+ * block scales passed through damoe_set_fp8_scales: weights one scale per 128x128 block,
+ * activations one per token and 128 consecutive channels; the value of an element is
+ * code * scale.  The intermediate h is rounded to bf16 and re-quantised on the device to E4M3
+ * with one scale per (pair, 128 channels): s = amax / 448 (1 when amax = 0), code =
+ * e4m3_rn_sat(h / s), both in fp32.  `out` is bf16.  FP8 contexts offer variants 0..3
+ * (N_v <= 128); a larger variant id is DAMOE_ERR_INVALID_ARG, and damoe_fused_moe_host is
+ * bf16 only.
  */
 int damoe_create(damoe_ctx** ctx, int device, int max_T, int k, int E, int H, int I, int dtype);
 int damoe_destroy(damoe_ctx* ctx);
@@ -153,8 +161,9 @@ int damoe_fused_moe_host(damoe_ctx* ctx, const void* x_host, const void* w13, co
                          int variant, void* out_host, void* stream);
 
 /* FP8 block scales (dtype == DAMOE_FP8_E4M3_BLOCK128 only): x_scale dev [T, H/128],
- * w13_scale dev [E, 2I/128, H/128], w2_scale dev [E, H/128, I/128], all float32.
- * Not implemented yet: returns DAMOE_ERR_UNSUPPORTED_SHAPE. */
+ * w13_scale dev [E, 2I/128, H/128], w2_scale dev [E, H/128, I/128], all float32, row-major.
+ * The pointers are remembered and read by every later damoe_fused_moe call on this context;
+ * x_scale must describe the `x` of that call. */
 int damoe_set_fp8_scales(damoe_ctx* ctx, const float* x_scale, const float* w13_scale,
                          const float* w2_scale);
 

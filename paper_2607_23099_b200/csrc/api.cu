@@ -35,6 +35,11 @@ struct damoe_ctx {
   CUtensorMap map_w13, map_w2;
   const void* cached_w13 = nullptr;
   const void* cached_w2 = nullptr;
+  // FP8 block scales set by damoe_set_fp8_scales (device pointers owned by the caller)
+  const float* x_scale = nullptr;
+  const float* w13_scale = nullptr;
+  const float* w2_scale = nullptr;
+  int num_variants() const { return dtype == DAMOE_BF16 ? kNumVariants : kNumVariantsFp8; }
   // staging for the host-buffer entry point
   void *st_x = nullptr, *st_ids = nullptr, *st_w = nullptr, *st_out = nullptr;
   // stage timing
@@ -78,15 +83,18 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// bf16 matrix [rows, cols] row-major, box = 64 columns (128 bytes) x box_rows, 128-byte swizzle.
+// Matrix [rows, cols] row-major of bf16 (or one-byte e4m3 codes), box = 128 bytes of columns x
+// box_rows, 128-byte swizzle.
 int make_map(damoe_ctx* c, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return fail(c, DAMOE_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+  const bool fp8 = c->dtype != DAMOE_BF16;
+  const uint64_t esize = fp8 ? 1 : 2;
   cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
-  cuuint32_t box[2] = {static_cast<cuuint32_t>(kBK), box_rows};
+  cuuint64_t strides[1] = {cols * esize};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(fp8 ? kBK8 : kBK), box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  CUresult r = fn(map, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(c, DAMOE_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
@@ -99,7 +107,7 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // expert's weights streamed from HBM, one extra pass served by L2, and tensor time per padded
 // token column with small tiles running the MMA pipe below peak.
 void default_cost_model(const damoe_ctx* c, int64_t* cost) {
-  const double wbytes = 3.0 * c->H * c->I * 2.0;
+  const double wbytes = 3.0 * c->H * c->I * (c->dtype == DAMOE_BF16 ? 2.0 : 1.0);
   const double flops_col = 6.0 * c->H * c->I;
   for (int v = 0; v < kNumVariants; ++v) {
     const int n = variant_desc(v).tile_n;
@@ -108,6 +116,7 @@ void default_cost_model(const damoe_ctx* c, int64_t* cost) {
     cost[1 * kNumVariants + v] = static_cast<int64_t>(wbytes / 6.5e12 * 1e12);
     cost[2 * kNumVariants + v] = static_cast<int64_t>(wbytes / 13e12 * 1e12);
     cost[3 * kNumVariants + v] = static_cast<int64_t>(flops_col / (1.4e15 * eff) * 1e12);
+    if (v >= c->num_variants()) cost[0 * kNumVariants + v] = 1ll << 36;  // not built for this dtype: never chosen
   }
 }
 
@@ -134,7 +143,7 @@ int make_selector(const damoe_ctx* c, int T, int variant, SelectorArgs* sel) {
   if (variant >= 0) {
     sel->forced = variant;
   } else if (variant == DAMOE_VARIANT_STATIC) {
-    sel->forced = b ? b->static_variant : kDefaultStaticVariant;
+    sel->forced = b ? b->static_variant : kDefaultStaticVariant;  // N = 64 exists for both dtypes
   } else if (b) {
     sel->mode = c->table_mode;
     sel->n_exemplars = b->n_ex;
@@ -199,7 +208,7 @@ int damoe_create(damoe_ctx** out, int device, int max_T, int k, int E, int H, in
   if (!out) return DAMOE_ERR_INVALID_ARG;
   *out = nullptr;
   if (max_T < 1 || k < 1 || E < 1 || H < 1 || I < 1) return DAMOE_ERR_INVALID_ARG;
-  if (dtype != DAMOE_BF16) return DAMOE_ERR_UNSUPPORTED_SHAPE;
+  if (dtype != DAMOE_BF16 && dtype != DAMOE_FP8_E4M3_BLOCK128) return DAMOE_ERR_UNSUPPORTED_SHAPE;
   if (k > kMaxK || E > kMaxE || H % 128 != 0 || I % 128 != 0) return DAMOE_ERR_UNSUPPORTED_SHAPE;
   if (static_cast<long long>(max_T) * k > 131072) return DAMOE_ERR_WORKSPACE;  // keeps the selector's integers in 64 bits
   damoe_ctx* c = new (std::nothrow) damoe_ctx();
@@ -215,7 +224,7 @@ int damoe_create(damoe_ctx** out, int device, int max_T, int k, int E, int H, in
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return bail(DAMOE_ERR_CUDA);
   if (prop.major != 10) return bail(DAMOE_ERR_UNSUPPORTED_SHAPE);  // tcgen05 kernels: sm_100a only
   c->sm_count = prop.multiProcessorCount;
-  if (gemm_configure() != cudaSuccess) return bail(DAMOE_ERR_CUDA);
+  if (gemm_configure() != cudaSuccess || gemm8_configure() != cudaSuccess) return bail(DAMOE_ERR_CUDA);
 
   // one arena; 1024-byte aligned slices
   const size_t P = c->max_P;
@@ -232,7 +241,9 @@ int damoe_create(damoe_ctx** out, int device, int max_T, int k, int E, int H, in
                o_tiles = carve(sizeof(int32_t) * kNumVariants),
                o_pref = carve(sizeof(int32_t) * kNumVariants * (E + 1)), o_act = carve(4), o_var = carve(4),
                o_stat = carve(4), o_bh = carve(sizeof(int32_t) * nblk * E), o_cost = carve(8 * 4 * kNumVariants),
-               o_xp = carve(2 * P * H), o_h = carve(2 * P * I), o_y = carve(4 * P * H),
+               o_xp = carve((dtype == DAMOE_BF16 ? 2 : 1) * P * H), o_h = carve((dtype == DAMOE_BF16 ? 2 : 1) * P * I),
+               o_xs = carve(dtype == DAMOE_BF16 ? 0 : 4 * P * (H / 128)), o_hs = carve(dtype == DAMOE_BF16 ? 0 : 4 * P * (I / 128)),
+               o_y = carve(4 * P * H),
                o_sx = carve(2 * static_cast<size_t>(max_T) * H), o_sid = carve(4 * P), o_sw = carve(4 * P),
                o_so = carve(2 * static_cast<size_t>(max_T) * H);
   if (cudaMalloc(&c->arena, off) != cudaSuccess) {
@@ -258,16 +269,25 @@ int damoe_create(damoe_ctx** out, int device, int max_T, int k, int E, int H, in
   c->ws.x_perm = reinterpret_cast<__nv_bfloat16*>(a + o_xp);
   c->ws.h = reinterpret_cast<__nv_bfloat16*>(a + o_h);
   c->ws.y = reinterpret_cast<float*>(a + o_y);
+  c->ws.xq_perm = a + o_xp;
+  c->ws.hq = a + o_h;
+  c->ws.xs_T = reinterpret_cast<float*>(a + o_xs);
+  c->ws.hs_T = reinterpret_cast<float*>(a + o_hs);
+  c->ws.max_P = c->max_P;
   c->st_x = a + o_sx; c->st_ids = a + o_sid; c->st_w = a + o_sw; c->st_out = a + o_so;
 
   int64_t cost[4 * kNumVariants];
   default_cost_model(c, cost);
   if (cudaMemcpy(c->default_cost, cost, sizeof(cost), cudaMemcpyHostToDevice) != cudaSuccess) return bail(DAMOE_ERR_CUDA);
 
-  for (int v = 0; v < kNumVariants; ++v) {
+  for (int v = 0; v < c->num_variants(); ++v) {
     const uint32_t n = variant_desc(v).tile_n;
     if (make_map(c, &c->map_x[v], c->ws.x_perm, P, H, n) != DAMOE_OK) return bail(DAMOE_ERR_CUDA);
     if (make_map(c, &c->map_h[v], c->ws.h, P, I, n) != DAMOE_OK) return bail(DAMOE_ERR_CUDA);
+  }
+  for (int v = c->num_variants(); v < kNumVariants; ++v) {
+    c->map_x[v] = c->map_x[0];
+    c->map_h[v] = c->map_h[0];
   }
   *out = c;
   return DAMOE_OK;
@@ -293,8 +313,14 @@ int damoe_set_dispatch(damoe_ctx* c, int mode) {
   return DAMOE_OK;
 }
 
-int damoe_set_fp8_scales(damoe_ctx* c, const float*, const float*, const float*) {
-  return fail(c, DAMOE_ERR_UNSUPPORTED_SHAPE, "FP8 block-scaled path is not implemented");
+int damoe_set_fp8_scales(damoe_ctx* c, const float* x_scale, const float* w13_scale, const float* w2_scale) {
+  if (!c) return DAMOE_ERR_INVALID_ARG;
+  if (c->dtype != DAMOE_FP8_E4M3_BLOCK128) return fail(c, DAMOE_ERR_INVALID_ARG, "context is not FP8");
+  if (!x_scale || !w13_scale || !w2_scale) return fail(c, DAMOE_ERR_INVALID_ARG, "null scale pointer");
+  c->x_scale = x_scale;
+  c->w13_scale = w13_scale;
+  c->w2_scale = w2_scale;
+  return DAMOE_OK;
 }
 
 int damoe_load_tuning_table(damoe_ctx* c, const void* bytes, size_t nbytes) {
@@ -318,7 +344,7 @@ int damoe_load_tuning_table(damoe_ctx* c, const void* bytes, size_t nbytes) {
     if (n) memcpy(blob.data() + o, src, n);
     return o;
   };
-  auto bad_variant = [&](int32_t v) { return v < 0 || v >= kNumVariants; };
+  auto bad_variant = [&](int32_t v) { return v < 0 || v >= c->num_variants(); };
   for (uint32_t i = 0; i < nb; ++i) {
     TableBucket& b = buckets[i];
     b.T = (int)r.get<uint32_t>();
@@ -354,6 +380,7 @@ int damoe_load_tuning_table(damoe_ctx* c, const void* bytes, size_t nbytes) {
     if (!r.ok) return fail(c, DAMOE_ERR_TABLE_FORMAT, "truncated bucket %u", i);
     for (int t = 0; t < 4 * kNumVariants; ++t)
       if (cost[t] < 0 || cost[t] > (1ll << 36)) return fail(c, DAMOE_ERR_TABLE_FORMAT, "cost out of range in bucket %u", i);
+    for (int v = c->num_variants(); v < kNumVariants; ++v) cost[v] = 1ll << 36;  // variants not built for this dtype
     b.off_ex = put(ex.data(), ex.size() * 4);
     b.off_exv = put(exv.data(), exv.size() * 4);
     b.off_bnum = put(bnum.data(), bnum.size() * 8);
@@ -401,7 +428,10 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
   if (T == 0) return DAMOE_OK;
   if (T < 0 || T > c->max_T) return fail(c, DAMOE_ERR_INVALID_ARG, "T=%d outside [0, %d]", T, c->max_T);
   if (!x || !w13 || !w2 || !topk_ids || !topk_weights || !out) return fail(c, DAMOE_ERR_INVALID_ARG, "null pointer");
-  if (variant >= kNumVariants || variant < DAMOE_VARIANT_STATIC) return fail(c, DAMOE_ERR_INVALID_ARG, "variant %d", variant);
+  if (variant >= c->num_variants() || variant < DAMOE_VARIANT_STATIC) return fail(c, DAMOE_ERR_INVALID_ARG, "variant %d", variant);
+  const bool fp8 = c->dtype != DAMOE_BF16;
+  if (fp8 && (!c->x_scale || !c->w13_scale || !c->w2_scale))
+    return fail(c, DAMOE_ERR_INVALID_ARG, "FP8 context: call damoe_set_fp8_scales first");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   DAMOE_CUDA(c, cudaSetDevice(c->device));
 
@@ -431,7 +461,10 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
   DAMOE_MARK(0);
   DAMOE_CUDA(c, launch_route(c->ws, topk_ids, topk_weights, T, c->k, c->E, sel, nullptr, nullptr, false, st));
   DAMOE_MARK(1);
-  DAMOE_CUDA(c, launch_gather(c->ws, static_cast<const __nv_bfloat16*>(x), T, c->k, c->H, st));
+  if (fp8)
+    DAMOE_CUDA(c, launch_gather8(c->ws, static_cast<const uint8_t*>(x), c->x_scale, T, c->k, c->H, st));
+  else
+    DAMOE_CUDA(c, launch_gather(c->ws, static_cast<const __nv_bfloat16*>(x), T, c->k, c->H, st));
   DAMOE_MARK(2);
 
   GemmMaps m13, m2;
@@ -451,7 +484,34 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
   ga.y = c->ws.y;
   ga.E = c->E; ga.H = c->H; ga.I = c->I;
 
-  if (known >= 0) {
+  GemmArgs8 g13{}, g2{};
+  g13.ntile_prefix = g2.ntile_prefix = c->ws.ntile_prefix;
+  g13.offsets = g2.offsets = c->ws.offsets;
+  g13.variant_id = g2.variant_id = c->ws.variant_id;
+  g13.status = g2.status = c->ws.status;
+  g13.w_sorted = g2.w_sorted = c->ws.w_sorted;
+  g13.hq = g2.hq = c->ws.hq;
+  g13.hs_T = g2.hs_T = c->ws.hs_T;
+  g13.y = g2.y = c->ws.y;
+  g13.E = g2.E = c->E; g13.H = g2.H = c->H; g13.I = g2.I = c->I; g13.max_P = g2.max_P = c->max_P;
+  g13.w_scale = c->w13_scale; g13.act_scale_T = c->ws.xs_T;
+  g2.w_scale = c->w2_scale; g2.act_scale_T = c->ws.hs_T;
+
+  if (fp8) {
+    if (known >= 0) {
+      DAMOE_CUDA(c, launch_gemm8(0, known, false, m13, g13, c->sm_count, st));
+      DAMOE_MARK(3);
+      DAMOE_CUDA(c, launch_gemm8(1, known, false, m2, g2, c->sm_count, st));
+    } else if (c->dispatch == DAMOE_DISPATCH_PREDICATED) {
+      for (int v = 0; v < kNumVariantsFp8; ++v) DAMOE_CUDA(c, launch_gemm8(0, v, true, m13, g13, c->sm_count, st));
+      DAMOE_MARK(3);
+      for (int v = 0; v < kNumVariantsFp8; ++v) DAMOE_CUDA(c, launch_gemm8(1, v, true, m2, g2, c->sm_count, st));
+    } else {
+      DAMOE_CUDA(c, launch_gemm8(0, -1, false, m13, g13, c->sm_count, st));
+      DAMOE_MARK(3);
+      DAMOE_CUDA(c, launch_gemm8(1, -1, false, m2, g2, c->sm_count, st));
+    }
+  } else if (known >= 0) {
     DAMOE_CUDA(c, launch_gemm(0, known, false, m13, ga, c->sm_count, st));
     DAMOE_MARK(3);
     DAMOE_CUDA(c, launch_gemm(1, known, false, m2, ga, c->sm_count, st));
@@ -478,6 +538,7 @@ int damoe_fused_moe_host(damoe_ctx* c, const void* x_host, const void* w13, cons
   if (T == 0) return DAMOE_OK;
   if (T < 0 || T > c->max_T) return fail(c, DAMOE_ERR_INVALID_ARG, "T=%d outside [0, %d]", T, c->max_T);
   if (!x_host || !topk_ids_host || !topk_weights_host || !out_host) return fail(c, DAMOE_ERR_INVALID_ARG, "null pointer");
+  if (c->dtype != DAMOE_BF16) return fail(c, DAMOE_ERR_UNSUPPORTED_SHAPE, "host-buffer entry point is bf16 only");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   DAMOE_CUDA(c, cudaSetDevice(c->device));
   const size_t P = static_cast<size_t>(T) * c->k;

@@ -63,6 +63,12 @@ struct Workspace {
   __nv_bfloat16* x_perm;    // [max_P, H]
   __nv_bfloat16* h;         // [max_P, I]
   float* y;                 // [max_P, H]
+  // FP8 contexts (dtype DAMOE_FP8_E4M3_BLOCK128) use these instead of x_perm / h
+  uint8_t* xq_perm;         // [max_P, H] e4m3 codes of the gathered activations
+  float* xs_T;              // [H/128, max_P] their 1x128 group scales, scale-block major
+  uint8_t* hq;              // [max_P, I] e4m3 codes of the re-quantised activation h
+  float* hs_T;              // [I/128, max_P] its 1x128 group scales, scale-block major
+  int max_P;
 };
 
 // route.cu
@@ -93,5 +99,27 @@ struct GemmArgs {
 cudaError_t launch_gemm(int kind, int variant, bool predicated, const GemmMaps& maps, const GemmArgs& args,
                         int sm_count, cudaStream_t stream);
 cudaError_t gemm_configure();  // opt-in shared-memory sizes, once per device
+
+// gemm_fp8.cu: the same family on kind::f8f6f4 with per-128-K-block scale promotion.
+constexpr int kNumVariantsFp8 = 4;  // N = 16, 32, 64, 128 (variant ids 0..3)
+constexpr int kBK8 = 128;           // K elements per stage = one 128x128 / 1x128 scale block
+struct GemmArgs8 {
+  const int32_t* ntile_prefix;
+  const int32_t* offsets;
+  const int32_t* variant_id;
+  uint32_t* status;
+  const float* w_scale;   // [E, rows/128, K/128]
+  const float* act_scale_T;  // [K/128, max_P]
+  const float* w_sorted;  // down GEMM only
+  uint8_t* hq;            // gate/up output codes [max_P, I]
+  float* hs_T;            // gate/up output scales [I/128, max_P]
+  float* y;               // down GEMM output [max_P, H]
+  int E, H, I, max_P;
+};
+cudaError_t launch_gemm8(int kind, int variant, bool predicated, const GemmMaps& maps, const GemmArgs8& args,
+                         int sm_count, cudaStream_t stream);
+cudaError_t gemm8_configure();
+cudaError_t launch_gather8(const Workspace& ws, const uint8_t* xq, const float* x_scale, int T, int k, int H,
+                           cudaStream_t stream);
 
 }  // namespace damoe

@@ -23,6 +23,7 @@
 // Every mbarrier wait is bounded; on a timeout the CTA raises DAMOE_STATUS_WAIT_TIMEOUT,
 // drains its outstanding TMA loads, frees its TMEM and returns.
 #include "common.cuh"
+#include "gemm_common.cuh"
 #include "ptx.cuh"
 
 namespace damoe {
@@ -49,32 +50,6 @@ struct Cfg {
   static_assert(kStageBytes % 1024 == 0, "operand tiles must stay 1024-byte aligned for the 128B swizzle");
   static_assert(kSmemBytes <= 232448, "over the 227 KB shared-memory limit");
 };
-
-struct Item {
-  int e, m_tile, q0, valid;
-};
-
-__device__ __forceinline__ Item decode_item(int w, const int* s_pref, const int* s_off, int E, int MT, int BN) {
-  int lo = 0, hi = E - 1;
-  while (lo < hi) {  // largest e with s_pref[e] * MT <= w
-    const int mid = (lo + hi + 1) >> 1;
-    if (s_pref[mid] * MT <= w) lo = mid;
-    else hi = mid - 1;
-  }
-  Item it;
-  it.e = lo;
-  const int nt = s_pref[lo + 1] - s_pref[lo];
-  const int local = w - s_pref[lo] * MT;
-  it.m_tile = local / nt;
-  const int n_tile = local - it.m_tile * nt;
-  const int off = s_off[lo];
-  it.q0 = off + n_tile * BN;
-  const int left = s_off[lo + 1] - it.q0;
-  it.valid = left < BN ? left : BN;
-  return it;
-}
-
-__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
 
 template <int KIND, int BN, int STAGES>
 __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUtensorMap* tmap_act, const GemmArgs& a,
@@ -162,10 +137,14 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(kTileM, BN);
       int it = 0, tile_i = 0;
       bool ok = true;
       for (int w = blockIdx.x; ok && w < total; w += gridDim.x, ++tile_i) {
+        // A ragged last token tile issues narrower MMAs: N is a field of the instruction
+        // descriptor, so only ceil16(valid) token columns cost tensor time.
+        const Item item = decode_item(w, s_pref, s_off, E, MT, BN);
+        const int n_eff = (item.valid + 15) & ~15;
+        const uint32_t idesc = umma_idesc_bf16(kTileM, n_eff < BN ? n_eff : BN);
         const int buf = tile_i % C::kNumAcc;
         const uint32_t aph = (tile_i / C::kNumAcc) & 1;
         if (!mbar_wait(bar_tempty + 8u * buf, aph ^ 1u, s_abort)) break;

@@ -1,0 +1,430 @@
+// Grouped expert GEMMs in FP8 (E4M3 x E4M3 -> fp32) on tcgen05 kind::f8f6f4 for sm_100a, with
+// fp32 block scales: weights carry one scale per 128x128 block, activations one per token and
+// 128 consecutive K.  The hardware block-scaled MMA wants 1x32 UE8M0 scales, which these are
+// not, so the scales are applied in software with a two-level accumulation: every K block of
+// 128 is multiplied into a TMEM partial accumulator (4 MMAs of K=32), and the epilogue warps
+// read the partial, multiply it by  w_scale[block] * act_scale[token, block]  and add it to
+// fp32 accumulators held in registers, while the MMA warp already fills the other partial
+// buffer.  Everything else follows the bf16 kernel: swap-AB, persistent CTAs decoding work
+// items from the device-side tile prefix, TMA-fed multistage ring, bounded waits.
+//
+// CTA = 10 warps: warp 0 TMA producer, warp 1 MMA issuer + TMEM allocation, warps 2..9
+// epilogue; epilogue warp pairs (w, w+4) share a TMEM lane quadrant and split the token
+// columns in halves, which keeps the register accumulators at N_v (gate/up) or N_v/2 (down)
+// floats per thread.
+//
+// KIND 0 (gate/up): a = silu(g) * u, h_b = bf16(a); the 128 channels of the weight tile are
+//   exactly one 1x128 scale group of h, so the group amax is a reduction over the tile's 128
+//   TMEM lanes: s = amax / 448 (1 when amax = 0), code = e4m3_rn_sat(h_b / s), both in fp32.
+// KIND 1 (down): y[q, m] = w_sorted[q] * acc, fp32.
+#include <cuda_fp8.h>
+
+#include "common.cuh"
+#include "gemm_common.cuh"
+#include "ptx.cuh"
+
+namespace damoe {
+
+namespace {
+
+constexpr int kThreads8 = 320;
+constexpr int kABytes8 = kTileM * kBK8;  // 128 rows x 128 one-byte elements
+constexpr int kTailBytes8 = 2 * (kMaxE + 1) * 4 + 512 + 2 * 4 * 128 * 4;  // + amax exchange, double-buffered [2][4 quadrants][BN <= 128]
+
+__device__ __forceinline__ void umma_fp8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// E4M3 A and B (format code 0), both K-major, fp32 accumulator, dense.
+__host__ __device__ constexpr uint32_t umma_idesc_e4m3(int M, int N) {
+  return (1u << 4) | (uint32_t(N >> 3) << 17) | (uint32_t(M >> 4) << 24);
+}
+
+template <int KIND, int BN, int STAGES>
+struct Cfg8 {
+  static constexpr int kATiles = (KIND == 0) ? 2 : 1;
+  static constexpr int kBBytes = BN * kBK8;
+  static constexpr int kStageBytes = kATiles * kABytes8 + kBBytes;
+  static constexpr int kAccCols = kATiles * BN;   // one partial buffer
+  static constexpr int kTmemColsRaw = 2 * kAccCols;
+  static constexpr int kTmemCols = kTmemColsRaw <= 32 ? 32 : kTmemColsRaw <= 64 ? 64 : kTmemColsRaw <= 128 ? 128
+                                   : kTmemColsRaw <= 256 ? 256 : 512;
+  static constexpr int kCW = BN / 2;              // token columns per epilogue warp
+  static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + kTailBytes8;
+  static_assert(kTmemColsRaw <= 512, "partials do not fit TMEM");
+  static_assert(kStageBytes % 1024 == 0, "operand tiles must stay 1024-byte aligned for the 128B swizzle");
+  static_assert(kSmemBytes <= 232448, "over the 227 KB shared-memory limit");
+};
+
+template <int CW>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float (&v)[CW]) {
+  if constexpr (CW == 8) {
+    uint32_t r[8];
+    tmem_ld_x8(taddr, r);
+    tmem_ld_wait();
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[j]);
+  } else {
+#pragma unroll
+    for (int c = 0; c < CW; c += 16) {
+      uint32_t r[16];
+      tmem_ld_x16(taddr + c, r);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 16; ++j) v[c + j] = __uint_as_float(r[j]);
+    }
+  }
+}
+
+template <int KIND, int BN, int STAGES>
+__device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUtensorMap* tmap_act, const GemmArgs8& a,
+                                           int variant, uint8_t* smem_raw) {
+  using C = Cfg8<KIND, BN, STAGES>;
+  constexpr int CW = C::kCW;
+  const int K = (KIND == 0) ? a.H : a.I;
+  const int MROWS = (KIND == 0) ? 2 * a.I : a.H;
+  const int MT = ((KIND == 0) ? a.I : a.H) / kTileM;
+  const int KB = K / kBK8;
+  const int E = a.E;
+
+  const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* tail = smem_raw + (tiles_base - smem_u32(smem_raw)) + STAGES * C::kStageBytes;
+  int* s_pref = reinterpret_cast<int*>(tail);
+  int* s_off = s_pref + (kMaxE + 1);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_off + (kMaxE + 1));
+  const uint32_t bar_full = smem_u32(bars);
+  const uint32_t bar_empty = bar_full + 8u * STAGES;
+  const uint32_t bar_pfull = bar_empty + 8u * STAGES;
+  const uint32_t bar_pempty = bar_pfull + 16u;
+  const uint32_t bar_xchg = bar_pempty + 16u;  // one per column half: the 4 warps sharing it exchange amax
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 6);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  float* s_amax = reinterpret_cast<float*>(s_tmem + 2);  // [2 buffers][4 quadrants][BN]
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  const int32_t* pref_g = a.ntile_prefix + variant * (E + 1);
+  for (int i = tid; i <= E; i += kThreads8) {
+    s_pref[i] = pref_g[i];
+    s_off[i] = a.offsets[i];
+  }
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_empty + 8u * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_pfull + 8u * b, 1);
+      mbar_init(bar_pempty + 8u * b, 8);
+      mbar_init(bar_xchg + 8u * b, 4);
+    }
+    *s_abort = 0;
+    fence_mbar_init();
+    fence_proxy_async_smem();
+    prefetch_tensormap(tmap_w);
+    prefetch_tensormap(tmap_act);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(s_tmem), C::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  const int total = s_pref[E] * MT;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int it = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
+        const Item item = decode_item(w, s_pref, s_off, E, MT, BN);
+        const int row_a = item.e * MROWS + item.m_tile * kTileM;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, s_abort)) {
+            ok = false;
+            break;
+          }
+          const uint32_t full = bar_full + 8u * s;
+          const uint32_t sa = tiles_base + s * C::kStageBytes;
+          mbar_arrive_expect_tx(full, C::kStageBytes);
+          tma_load_2d(sa, tmap_w, full, kb * kBK8, row_a);
+          if (KIND == 0) tma_load_2d(sa + kABytes8, tmap_w, full, kb * kBK8, row_a + a.I);
+          tma_load_2d(sa + C::kATiles * kABytes8, tmap_act, full, kb * kBK8, item.q0);
+        }
+      }
+      if (!ok) {
+        int dummy = 0;
+        for (int j = (it > STAGES ? it - STAGES : 0); j < it; ++j)
+          mbar_wait(bar_full + 8u * (j % STAGES), (j / STAGES) & 1, &dummy, 200000000ull);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: one partial accumulator per K block of 128 ----------------
+    if (lane == 0) {
+      int it = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
+        const Item item = decode_item(w, s_pref, s_off, E, MT, BN);
+        const int n_eff = (item.valid + 15) & ~15;
+        const uint32_t idesc = umma_idesc_e4m3(kTileM, n_eff < BN ? n_eff : BN);
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          const int pb = it & 1;
+          const uint32_t pph = (it >> 1) & 1;
+          if (!mbar_wait(bar_pempty + 8u * pb, pph ^ 1u, s_abort) || !mbar_wait(bar_full + 8u * s, ph, s_abort)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t sa = tiles_base + s * C::kStageBytes;
+          const uint64_t da0 = umma_desc_sw128(sa);
+          const uint64_t da1 = umma_desc_sw128(sa + kABytes8);
+          const uint64_t db = umma_desc_sw128(sa + C::kATiles * kABytes8);
+          const uint32_t d0 = tmem_base + pb * C::kAccCols;
+#pragma unroll
+          for (int k = 0; k < kBK8 / 32; ++k) {  // K = 32 per instruction = 32 bytes
+            umma_fp8(d0, da0 + 2u * k, db + 2u * k, idesc, k ? 1u : 0u);
+            if (KIND == 0) umma_fp8(d0 + BN, da1 + 2u * k, db + 2u * k, idesc, k ? 1u : 0u);
+          }
+          umma_commit(bar_empty + 8u * s);
+          umma_commit(bar_pfull + 8u * pb);
+        }
+      }
+    }
+  } else {
+    // ---------------- epilogue warps: scale promotion, then the fused output ----------------
+    const int ew = warp - 2;                        // 0..7
+    const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
+    const int half = ew >> 2;                       // which half of the token columns
+    const uint32_t lane_base = quad * 32;
+    const int col0 = half * CW;
+    const int wblocks_k = K / 128;
+    const float* wsc = a.w_scale;
+    int it = 0, item_i = 0;
+    for (int w = blockIdx.x; w < total; w += gridDim.x, ++item_i) {
+      const Item item = decode_item(w, s_pref, s_off, E, MT, BN);
+      const int ch = item.m_tile * kTileM + lane_base + lane;
+      // weight-scale rows of this item: [expert, row block, K block]
+      const float* wg = wsc + (static_cast<size_t>(item.e) * (MROWS / 128) + item.m_tile) * wblocks_k;
+      const float* wu = (KIND == 0) ? wg + static_cast<size_t>(a.I / 128) * wblocks_k : wg;
+      float acc_g[CW], acc_u[(KIND == 0) ? CW : 1];
+#pragma unroll
+      for (int j = 0; j < CW; ++j) acc_g[j] = 0.f;
+      if (KIND == 0) {
+#pragma unroll
+        for (int j = 0; j < CW; ++j) acc_u[j] = 0.f;
+      }
+      bool ok = true;
+      for (int kb = 0; kb < KB; ++kb, ++it) {
+        const int pb = it & 1;
+        const uint32_t pph = (it >> 1) & 1;
+        // this lane's share of the activation scales of the K block: lane l holds column col0+l (and +32)
+        const float* xs = a.act_scale_T + static_cast<size_t>(kb) * a.max_P + item.q0 + col0;
+        float sx0 = 0.f, sx1 = 0.f;
+        if (lane < CW && col0 + lane < item.valid) sx0 = __ldg(xs + lane);
+        if (CW > 32 && col0 + 32 + lane < item.valid) sx1 = __ldg(xs + 32 + lane);
+        const float swg = __ldg(wg + kb);
+        const float swu = (KIND == 0) ? __ldg(wu + kb) : 0.f;
+        if (!mbar_wait(bar_pfull + 8u * pb, pph, s_abort)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t t0 = tmem_base + (lane_base << 16) + pb * C::kAccCols + col0;
+        if (col0 < item.valid) {
+          float p[CW];
+          tmem_ld_cols<CW>(t0, p);
+#pragma unroll
+          for (int j = 0; j < CW; ++j) {
+            const float sx = __shfl_sync(0xffffffffu, (j < 32) ? sx0 : sx1, j & 31);
+            acc_g[j] = fmaf(p[j], sx * swg, acc_g[j]);
+          }
+          if (KIND == 0) {
+            tmem_ld_cols<CW>(t0 + BN, p);
+#pragma unroll
+            for (int j = 0; j < CW; ++j) {
+              const float sx = __shfl_sync(0xffffffffu, (j < 32) ? sx0 : sx1, j & 31);
+              acc_u[j] = fmaf(p[j], sx * swu, acc_u[j]);
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_pempty + 8u * pb);
+      }
+      if (!ok) break;
+      if (KIND == 0) {
+        // h_b = bf16(silu(g) * u); group amax over the tile's 128 channels (= 128 TMEM lanes)
+        // The exchange buffer alternates per item; a warp can only reach item i+2 after all four
+        // warps of its half have arrived at item i+1's exchange, i.e. after they read item i's.
+        float* xa = s_amax + (item_i & 1) * 4 * BN;
+        float hb[CW];
+#pragma unroll
+        for (int j = 0; j < CW; ++j) {
+          hb[j] = __bfloat162float(__float2bfloat16_rn(silu_mul(acc_g[j], acc_u[j])));
+          const unsigned m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(hb[j])));
+          if (lane == 0) xa[quad * BN + col0 + j] = __uint_as_float(m);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_xchg + 8u * half);
+        if (!mbar_wait(bar_xchg + 8u * half, item_i & 1, s_abort)) break;   // bounded, like every wait here
+#pragma unroll
+        for (int j = 0; j < CW; ++j) {
+          const int n = col0 + j;
+          if (n < item.valid) {
+            const float amax = fmaxf(fmaxf(xa[0 * BN + n], xa[1 * BN + n]), fmaxf(xa[2 * BN + n], xa[3 * BN + n]));
+            const float sc = (amax == 0.f) ? 1.0f : __fdiv_rn(amax, 448.0f);
+            const uint8_t code = static_cast<uint8_t>(__nv_cvt_float_to_fp8(__fdiv_rn(hb[j], sc), __NV_SATFINITE, __NV_E4M3));
+            a.hq[static_cast<size_t>(item.q0 + n) * a.I + ch] = code;
+            if (quad == 0 && lane == 0) a.hs_T[static_cast<size_t>(item.m_tile) * a.max_P + item.q0 + n] = sc;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < CW; ++j) {
+          const int n = col0 + j;
+          if (n < item.valid)
+            a.y[static_cast<size_t>(item.q0 + n) * a.H + ch] = __ldg(a.w_sorted + item.q0 + n) * acc_g[j];
+        }
+      }
+    }
+  }
+
+  // ---------------- teardown ----------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem_base, C::kTmemCols);
+  }
+  if (tid == 0 && *s_abort) atomicOr(a.status, DAMOE_STATUS_WAIT_TIMEOUT);
+}
+
+__host__ __device__ constexpr int stages8(int kind, int v) {
+  constexpr int s13[kNumVariantsFp8] = {6, 5, 5, 4};
+  constexpr int s2[kNumVariantsFp8] = {10, 10, 8, 6};
+  return kind == 0 ? s13[v] : s2[v];
+}
+
+template <int KIND, int V>
+struct VCfg8 {
+  static constexpr int kBN = variant_desc(V).tile_n;
+  static constexpr int kStages = stages8(KIND, V);
+  using C = Cfg8<KIND, kBN, kStages>;
+};
+
+template <int KIND, int V>
+__global__ void __launch_bounds__(kThreads8, 1)
+    gemm8_fixed_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_act,
+                       const GemmArgs8 a, const int predicated) {
+  extern __shared__ uint8_t smem_raw[];
+  if (predicated && *a.variant_id != V) return;
+  gemm8_body<KIND, VCfg8<KIND, V>::kBN, VCfg8<KIND, V>::kStages>(&tmap_w, &tmap_act, a, V, smem_raw);
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(kThreads8, 1)
+    gemm8_branch_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs8 a) {
+  extern __shared__ uint8_t smem_raw[];
+  const int v = *a.variant_id;
+  switch (v) {
+    case 0: gemm8_body<KIND, VCfg8<KIND, 0>::kBN, VCfg8<KIND, 0>::kStages>(&maps.w, &maps.act[0], a, 0, smem_raw); break;
+    case 1: gemm8_body<KIND, VCfg8<KIND, 1>::kBN, VCfg8<KIND, 1>::kStages>(&maps.w, &maps.act[1], a, 1, smem_raw); break;
+    case 2: gemm8_body<KIND, VCfg8<KIND, 2>::kBN, VCfg8<KIND, 2>::kStages>(&maps.w, &maps.act[2], a, 2, smem_raw); break;
+    case 3: gemm8_body<KIND, VCfg8<KIND, 3>::kBN, VCfg8<KIND, 3>::kStages>(&maps.w, &maps.act[3], a, 3, smem_raw); break;
+    default: break;
+  }
+}
+
+template <int KIND>
+constexpr int max_smem8() {
+  int m = VCfg8<KIND, 0>::C::kSmemBytes;
+  m = VCfg8<KIND, 1>::C::kSmemBytes > m ? VCfg8<KIND, 1>::C::kSmemBytes : m;
+  m = VCfg8<KIND, 2>::C::kSmemBytes > m ? VCfg8<KIND, 2>::C::kSmemBytes : m;
+  m = VCfg8<KIND, 3>::C::kSmemBytes > m ? VCfg8<KIND, 3>::C::kSmemBytes : m;
+  return m;
+}
+
+template <int KIND, int V>
+cudaError_t launch_fixed8(const GemmMaps& maps, const GemmArgs8& args, bool predicated, int grid, cudaStream_t st) {
+  gemm8_fixed_kernel<KIND, V><<<grid, kThreads8, VCfg8<KIND, V>::C::kSmemBytes, st>>>(maps.w, maps.act[V], args,
+                                                                                      predicated ? 1 : 0);
+  return cudaGetLastError();
+}
+
+template <int KIND>
+cudaError_t launch_kind8(int variant, bool predicated, const GemmMaps& maps, const GemmArgs8& args, int grid,
+                         cudaStream_t st) {
+  switch (variant) {
+    case -1:
+      gemm8_branch_kernel<KIND><<<grid, kThreads8, max_smem8<KIND>(), st>>>(maps, args);
+      return cudaGetLastError();
+    case 0: return launch_fixed8<KIND, 0>(maps, args, predicated, grid, st);
+    case 1: return launch_fixed8<KIND, 1>(maps, args, predicated, grid, st);
+    case 2: return launch_fixed8<KIND, 2>(maps, args, predicated, grid, st);
+    case 3: return launch_fixed8<KIND, 3>(maps, args, predicated, grid, st);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+// xq_perm[q, :] = xq[perm[q] / k, :], xs_T[b, q] = x_scale[perm[q] / k, b]
+__global__ void __launch_bounds__(256) gather_rows8_kernel(const uint4* __restrict__ xq, const float* __restrict__ xs,
+                                                           uint4* __restrict__ xq_perm, float* __restrict__ xs_T,
+                                                           const int32_t* __restrict__ perm, int k, int row_vec,
+                                                           int nblk, int max_P) {
+  const int q = blockIdx.x;
+  const int p = perm[q];
+  if (p < 0) return;
+  const int t = p / k;
+  const uint4* src = xq + static_cast<size_t>(t) * row_vec;
+  uint4* dst = xq_perm + static_cast<size_t>(q) * row_vec;
+  for (int i = threadIdx.x; i < row_vec; i += blockDim.x) dst[i] = __ldg(src + i);
+  for (int b = threadIdx.x; b < nblk; b += blockDim.x) xs_T[static_cast<size_t>(b) * max_P + q] = xs[static_cast<size_t>(t) * nblk + b];
+}
+
+}  // namespace
+
+cudaError_t gemm8_configure() {
+  cudaError_t e;
+#define DAMOE_CFG8(K, V)                                                                                    \
+  if ((e = cudaFuncSetAttribute(gemm8_fixed_kernel<K, V>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                                VCfg8<K, V>::C::kSmemBytes)) != cudaSuccess)                                \
+    return e;
+  DAMOE_CFG8(0, 0) DAMOE_CFG8(0, 1) DAMOE_CFG8(0, 2) DAMOE_CFG8(0, 3)
+  DAMOE_CFG8(1, 0) DAMOE_CFG8(1, 1) DAMOE_CFG8(1, 2) DAMOE_CFG8(1, 3)
+#undef DAMOE_CFG8
+  if ((e = cudaFuncSetAttribute(gemm8_branch_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem8<0>())) !=
+      cudaSuccess)
+    return e;
+  return cudaFuncSetAttribute(gemm8_branch_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem8<1>());
+}
+
+cudaError_t launch_gemm8(int kind, int variant, bool predicated, const GemmMaps& maps, const GemmArgs8& args,
+                         int sm_count, cudaStream_t stream) {
+  return kind == 0 ? launch_kind8<0>(variant, predicated, maps, args, sm_count, stream)
+                   : launch_kind8<1>(variant, predicated, maps, args, sm_count, stream);
+}
+
+cudaError_t launch_gather8(const Workspace& ws, const uint8_t* xq, const float* x_scale, int T, int k, int H,
+                           cudaStream_t stream) {
+  gather_rows8_kernel<<<T * k, 256, 0, stream>>>(reinterpret_cast<const uint4*>(xq), x_scale,
+                                                 reinterpret_cast<uint4*>(ws.xq_perm), ws.xs_T, ws.perm, k, H / 16,
+                                                 H / 128, ws.max_P);
+  return cudaGetLastError();
+}
+
+}  // namespace damoe

@@ -1,0 +1,116 @@
+"""FP8 (E4M3, 128x128 / 1x128 fp32 block scales) path against the fp64 oracle on the same
+quantised inputs: integer outputs bit-exact, layer output within relative Frobenius 2e-2."""
+import numpy as np
+import pytest
+import torch
+
+import damoe_inputs as di
+from helpers import bits16, rel_frobenius
+from oracle import codecs, layer, route
+
+pytestmark = pytest.mark.gpu
+
+FROB_TOL_FP8 = 2e-2
+
+
+@pytest.fixture(scope="module")
+def d():
+    import paper_2607_23099_b200 as d
+    return d
+
+
+class Fp8Case:
+    def __init__(self, seed, T, E, k, H, I, alpha, weights=None):
+        self.T, self.E, self.k, self.H, self.I = T, E, k, H, I
+        self.ids, self.w, _ = di.routing_batch(seed, T, k, E, alpha)
+        self.W = weights or di.MoEWeights(77, E, H, I)
+        dev = "cuda:0"
+        self.xq, self.xs = di.quantize_e4m3_blocks(di.activations(seed, T, H, dev), 1, 128)
+        self.ids_d = torch.from_numpy(self.ids).to(dev)
+        self.w_d = torch.from_numpy(self.w).to(dev)
+
+
+def _run(d, m, case, wq, variant):
+    w13q, w13s, w2q, w2s = wq
+    m._check(d._lib.damoe_set_fp8_scales(m._ctx, d._ptr(case.xs), d._ptr(w13s), d._ptr(w2s)))
+    out = m.fused_moe(case.xq, w13q, w2q, case.ids_d, case.w_d, variant)
+    meta = m.debug_fetch(case.T)
+    return out, meta
+
+
+def _oracle(case, wq, tokens=None):
+    w13q, w13s, w2q, w2s = wq
+    np_ = lambda t: t.cpu().numpy()
+    bits, _ = layer.moe_layer_fp8(np_(case.xq), np_(case.xs), lambda e: np_(w13q[e]), lambda e: np_(w13s[e]),
+                                  lambda e: np_(w2q[e]), lambda e: np_(w2s[e]), case.ids, case.w, case.E, tokens=tokens)
+    return codecs.bf16_decode(bits)
+
+
+def _check(out, ref, tokens=None):
+    got = codecs.bf16_decode(bits16(out))
+    if tokens is not None:
+        got = got[np.asarray(tokens)]
+    fro = rel_frobenius(got, ref)
+    assert np.all(np.isfinite(got))
+    assert fro <= FROB_TOL_FP8, f"relative Frobenius {fro}"
+    return fro
+
+
+def test_fp8_tiny_every_variant(d):
+    case = Fp8Case(0, 64, 8, 2, 1024, 512, 1.0)
+    wq = case.W.materialize_fp8("cuda:0")
+    m = d.DAMoE(64, 2, 8, 1024, 512, dtype=d.FP8_E4M3_BLOCK128)
+    ref = _oracle(case, wq)
+    for variant in [0, 1, 2, 3, d.VARIANT_AUTO, d.VARIANT_STATIC]:
+        out, meta = _run(d, m, case, wq, variant)
+        assert meta["status"] == 0
+        off, perm, inv = route.offsets_and_permutation(case.ids, case.E)
+        assert np.array_equal(meta["offsets"], off) and np.array_equal(meta["inv"], inv)
+        _check(out, ref)
+    with pytest.raises(d.DamoeError):
+        _run(d, m, case, wq, 4)                       # N = 256 is not built for FP8
+    m.set_dispatch(d.DISPATCH_PREDICATED)
+    out, meta = _run(d, m, case, wq, d.VARIANT_AUTO)
+    assert meta["status"] == 0
+    _check(out, ref)
+    m.close()
+
+
+def test_fp8_ragged_multi_tile(d):
+    case = Fp8Case(5, 300, 8, 2, 1024, 512, 0.3)
+    wq = case.W.materialize_fp8("cuda:0")
+    m = d.DAMoE(512, 2, 8, 1024, 512, dtype=d.FP8_E4M3_BLOCK128)
+    ref = _oracle(case, wq)
+    for variant in range(4):
+        out, meta = _run(d, m, case, wq, variant)
+        assert meta["status"] == 0
+        _check(out, ref)
+        out2, _ = _run(d, m, case, wq, variant)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
+    m.close()
+
+
+def test_fp8_scales_are_required(d):
+    case = Fp8Case(1, 4, 8, 2, 1024, 512, 1.0)
+    wq = case.W.materialize_fp8("cuda:0")
+    m = d.DAMoE(8, 2, 8, 1024, 512, dtype=d.FP8_E4M3_BLOCK128)
+    with pytest.raises(d.DamoeError):
+        m.fused_moe(case.xq, wq[0], wq[2], case.ids_d, case.w_d, 0)
+    m.close()
+
+
+def test_fp8_config4_shape_sampled_tokens(d):
+    E, k, H, I = 256, 8, 7168, 2048
+    W = di.MoEWeights(12345, E, H, I)
+    wq = W.materialize_fp8("cuda:0")
+    m = d.DAMoE(256, k, E, H, I, dtype=d.FP8_E4M3_BLOCK128)
+    for T, alpha, seed, variant in [(16, 0.1, 0, d.VARIANT_AUTO), (256, 10.0, 1, 1), (256, 1.0, 2, 3)]:
+        case = Fp8Case(seed, T, E, k, H, I, alpha, weights=W)
+        out, meta = _run(d, m, case, wq, variant)
+        assert meta["status"] == 0
+        hist = route.histogram(case.ids, E)
+        assert np.array_equal(meta["tiles"], route.tile_counts(hist, d.tile_ns()))
+        tokens = [int(v) for v in np.random.default_rng(seed).choice(T, size=2, replace=False)]
+        _check(out, _oracle(case, wq, tokens=tokens), tokens=tokens)
+    m.close()
