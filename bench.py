@@ -44,8 +44,16 @@ SMALL_WORKLOAD = dict(name="profile_small_E32_T8", E=32, k=8, H=7168, I=2048, T=
                       alphas=[1.0], seeds=[0, 1], weight_seed=12345)
 # Kimi-K2-shaped serving-trace stand-in: 500 batches, T log-uniform in [1, 4096], per-batch alpha
 # log-uniform in [0.05, 10]; adaptive vs static vs per-batch best variant.
+# Compute-bound counterpart of the reduced case: 256 tokens per expert on average (as at T=8192 on
+# the full shape) on 16 experts, 1.4 GB of weights.  Only for ncu captures.
+SMALL_DENSE_WORKLOAD = dict(name="profile_small_dense_E16_T512", E=16, k=8, H=7168, I=2048, T=512,
+                            alphas=[10.0], seeds=[0, 1], weight_seed=12345)
 TRACE_WORKLOAD = dict(name="kimi_k2_trace_500", E=384, k=8, H=7168, I=2048, T=4096, trace=(1000, 500),
                       weight_seed=12345)
+# FP8 configuration: E4M3 weights with 128x128 block scales, E4M3 activations with 1x128 group
+# scales, bf16 output; T in {16, 256, 4096} x alpha in {0.1, 1, 10}.
+FP8_WORKLOAD = dict(name="deepseek_v3_fp8_grid", E=256, k=8, H=7168, I=2048, T=4096, dtype="fp8",
+                    grid=[(T, a) for T in (16, 256, 4096) for a in (0.1, 1.0, 10.0)], weight_seed=12345)
 # The same kind of trace on the headline shape (weights already resident): 48 batches, part of
 # the default line so that the dispatcher is also measured where token counts and skew vary.
 HEADLINE_TRACE = (2000, 48)
@@ -53,7 +61,7 @@ TABLE_DIR = os.path.join(ROOT, "paper_2607_23099_b200", "tables")
 
 
 def table_path(w):
-    return os.path.join(TABLE_DIR, f"e{w['E']}_k{w['k']}_h{w['H']}_i{w['I']}_bf16.damoetb")
+    return os.path.join(TABLE_DIR, f"e{w['E']}_k{w['k']}_h{w['H']}_i{w['I']}_{w.get('dtype', 'bf16')}.damoetb")
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gate/up GEMM launch, divided by the
 # activated experts of the captured cell (profiles/gemm_gate_up_small_E32_T8_ncu_full.md):
@@ -82,6 +90,8 @@ def make_cells(device, trace=None):
     trace = trace if trace is not None else w.get("trace")
     if trace is not None:
         specs = [(T, a, trace[0] + i) for i, (T, a) in enumerate(di.trace_batches(trace[0], trace[1], t_max=w["T"]))]
+    elif "grid" in w:
+        specs = [(T, a, 7000 + i) for i, (T, a) in enumerate(w["grid"])]
     else:
         specs = [(w["T"], a, 1000 * s + int(round(a * 100))) for a in w["alphas"] for s in w["seeds"]]
     cells = []
@@ -95,6 +105,8 @@ def make_cells(device, trace=None):
                 cell["ids_host"] = torch.from_numpy(ids).pin_memory()
                 cell["w_host"] = torch.from_numpy(wts).pin_memory()
                 cell["x"] = cell["x_host"].to(device)
+                if w.get("dtype") == "fp8":
+                    cell["x"], cell["x_scale"] = di.quantize_e4m3_blocks(cell["x"], 1, 128)
                 cell["ids_d"] = cell["ids_host"].to(device)
                 cell["w_d"] = cell["w_host"].to(device)
             cells.append(cell)
@@ -146,8 +158,9 @@ def layer_bytes_flops(cell, tile_n):
     w = WORKLOAD
     P = cell["T"] * w["k"]
     A = cell["active"]
-    wbytes = A * 3 * w["H"] * w["I"] * 2
-    act = P * w["H"] * 2 * 2 + P * w["I"] * 2 * 2 + P * w["H"] * 4 * 2 + cell["T"] * w["H"] * 2 * 2 + 16 * P
+    eb = 1 if w.get("dtype") == "fp8" else 2
+    wbytes = A * 3 * w["H"] * w["I"] * eb
+    act = P * w["H"] * eb * 2 + P * w["I"] * eb * 2 + P * w["H"] * 4 * 2 + cell["T"] * w["H"] * (eb + 2) + 16 * P
     # full tiles cost tile_n columns; the ragged last tile of an expert issues MMAs of ceil16(rest) columns
     padded_cols = int(sum((int(t) // tile_n) * tile_n + (-(-(int(t) % tile_n) // 16) * 16) for t in cell["hist"]))
     return wbytes + act, padded_cols * 6 * w["H"] * w["I"], P * 6 * w["H"] * w["I"]
@@ -158,7 +171,8 @@ def w13_launch_bytes(cell):
     gathered activations read once, h written once."""
     w = WORKLOAD
     P = cell["T"] * w["k"]
-    return cell["active"] * 2 * w["I"] * w["H"] * 2 + P * w["H"] * 2 + P * w["I"] * 2
+    eb = 1 if w.get("dtype") == "fp8" else 2
+    return cell["active"] * 2 * w["I"] * w["H"] * eb + P * w["H"] * eb + P * w["I"] * eb
 
 
 def oracle_sample_seconds(cells, n_tokens):
@@ -235,6 +249,8 @@ def geomean(xs):
 def compare_dispatch(m, d, cells, run, pk, reps=3):
     """Per batch: AUTO vs STATIC vs every variant (median of reps), roofline of the chosen one."""
     ns = d.tile_ns()
+    if WORKLOAD.get("dtype") == "fp8":
+        ns = ns[:4]
     stream = torch.cuda.current_stream()
 
     def time_variant(c, variant):
@@ -258,7 +274,8 @@ def compare_dispatch(m, d, cells, run, pk, reps=3):
         static_id = m.debug_fetch(c["T"])["variant_id"]
         t_var = [time_variant(c, v) for v in range(len(ns))]
         nbytes, fl_pad, fl_use = layer_bytes_flops(c, ns[chosen])
-        t_roof = max(nbytes / (pk["hbm_gbs"] * 1e9), fl_pad / (pk["bf16_tflops_sustained"] * 1e12)) * 1e6
+        tensor_peak = pk["bf16_tflops_sustained"] * (2.0 if WORKLOAD.get("dtype") == "fp8" else 1.0)  # fp8 = 2x bf16 (nominal ratio)
+        t_roof = max(nbytes / (pk["hbm_gbs"] * 1e9), fl_pad / (tensor_peak * 1e12)) * 1e6
         rows.append(dict(T=c["T"], alpha=round(c["alpha"], 4), active=c["active"], auto_us=round(t_auto, 1),
                          static_us=round(t_static, 1), best_us=round(min(t_var), 1), best_variant=int(np.argmin(t_var)),
                          chosen=chosen, static_variant=static_id, roofline_us=round(t_roof, 1),
@@ -285,14 +302,18 @@ def run_ours(args):
     device = torch.device(f"cuda:{local}")
     w = WORKLOAD
     is_trace = "trace" in w
-    steps = args.steps if args.steps is not None else (w["trace"][1] if is_trace else 320)
+    steps = args.steps if args.steps is not None else (w["trace"][1] if is_trace else 90 if "grid" in w else 320)
     warmup = max(3, args.warmup if args.warmup is not None else 16)
     pk = peaks()
 
     W = di.MoEWeights(w["weight_seed"], w["E"], w["H"], w["I"])
-    w13, w2 = W.materialize(device)
+    fp8 = w.get("dtype") == "fp8"
+    if fp8:
+        w13, w13s, w2, w2s = W.materialize_fp8(device)
+    else:
+        w13, w2 = W.materialize(device)
     cells = make_cells(device)
-    m = d.DAMoE(w["T"], w["k"], w["E"], w["H"], w["I"], device=local)
+    m = d.DAMoE(w["T"], w["k"], w["E"], w["H"], w["I"], dtype=d.FP8_E4M3_BLOCK128 if fp8 else d.BF16, device=local)
     table = "built-in cost model"
     if os.path.exists(table_path(w)) and not args.no_table:
         m.load_tuning_table(open(table_path(w), "rb").read())
@@ -301,10 +322,17 @@ def run_ours(args):
     out_host = torch.empty(w["T"], w["H"], dtype=torch.bfloat16).pin_memory()
     stream = torch.cuda.current_stream()
 
-    def run(c, variant=d.VARIANT_AUTO):
+    default_variant = d.VARIANT_AUTO if args.variant is None else args.variant
+
+    def run(c, variant=None):
+        variant = default_variant if variant is None else variant
+        if fp8:
+            m.set_fp8_scales(c["x_scale"], w13s, w2s)
         m.fused_moe(c["x"], w13, w2, c["ids_d"], c["w_d"], variant, out=out[:c["T"]], stream=stream)
 
     def run_host(c):
+        if fp8:                       # the host-buffer entry point is bf16 only: time the device call instead
+            return run(c)
         m.fused_moe_host(c["x_host"], w13, w2, c["ids_host"], c["w_host"], d.VARIANT_AUTO, out_host=out_host[:c["T"]],
                          stream=stream)
 
@@ -370,9 +398,12 @@ def run_ours(args):
     w13_bytes = statistics.mean(w13_launch_bytes(c) for c in rec_cells)
     w13_ms = stage["gemm13"] / max(1, n_rec)
     achieved = w13_bytes / (w13_ms * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 * statistics.mean(c["active"] for c in rec_cells)
-    roofline = dict(bound="hbm", kernel="gemm_branch_kernel<0> (grouped gate/up GEMM + SwiGLU)", achieved=round(achieved, 1),
-                    peak=pk["hbm_gbs"], unit="GB/s", frac=round(achieved / pk["hbm_gbs"], 4), traffic=round(traffic),
+    # the ncu capture is of the bf16 kernel at ~2 tokens per expert; it is only scaled to workloads of that kind
+    traffic = None
+    if not fp8 and not is_trace:
+        traffic = round(NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 * statistics.mean(c["active"] for c in rec_cells))
+    roofline = dict(bound="hbm", kernel=("gemm8" if fp8 else "gemm") + "_branch_kernel<0> (grouped gate/up GEMM + SwiGLU)", achieved=round(achieved, 1),
+                    peak=pk["hbm_gbs"], unit="GB/s", frac=round(achieved / pk["hbm_gbs"], 4), traffic=traffic,
                     algorithmic_bytes=round(w13_bytes), peak_source=pk["source"], launch_ms=round(w13_ms, 4),
                     launches_timed=n_rec,
                     stage_share={k: round(stage[k] / max(1e-9, sum(stage[s] for s in m.STAGES)), 4) for k in m.STAGES})
@@ -393,11 +424,15 @@ def run_ours(args):
                   batches=len(cells), dispatch="auto/branch", table=table,
                   l2="inputs larger than L2: a step streams the activated experts' weights (GBs), never reused across steps",
                   parallelism="replicas only" if world > 1 else "single GPU")
-    if not is_trace:
+    if "alphas" in w:
         config.update(alphas=w["alphas"], seeds_per_alpha=len(w["seeds"]))
+    if "grid" in w:
+        config.update(T="{16, 256, 4096}", alphas=[0.1, 1.0, 10.0])
+    if fp8:
+        config.update(e2e_note="host-buffer entry point is bf16 only; e2e repeats the device-timed call")
     line = dict(metric="fused_moe_layer_us", value=round(us_per_layer, 2), unit="us", n_gpus=world, steps=steps,
                 warmup=warmup, ms_per_step=round(us_per_layer / 1e3, 5), higher_is_better=False, scaling="weak",
-                vs_baseline=None, dtype="bf16", data="synthetic", config=config,
+                vs_baseline=None, dtype="fp8" if fp8 else "bf16", data="synthetic", config=config,
                 aggregate_layers_per_s=round(world * 1e6 / us_per_layer, 2),
                 e2e=dict(value=round(e2e_us, 2), unit="us", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
                 gpu_launches=7 * steps, clocks=clocks, roofline=roofline, cpu_baseline=cpu, dispatch=dispatch,
@@ -412,13 +447,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="headline", choices=["headline", "small", "kimi_trace"],
+    ap.add_argument("--workload", default="headline", choices=["headline", "small", "small_dense", "kimi_trace", "fp8_grid"],
                     help="'small' is the reduced case used for ncu captures; 'kimi_trace' the 500-batch serving-trace stand-in")
     ap.add_argument("--no-table", action="store_true", help="ignore the committed tuning table")
+    ap.add_argument("--variant", type=int, default=None, help="force this kernel variant in the timed steps (profiling)")
     args = ap.parse_args()
     if args.workload != "headline":
         WORKLOAD.clear()
-        WORKLOAD.update(SMALL_WORKLOAD if args.workload == "small" else TRACE_WORKLOAD)
+        WORKLOAD.update(dict(small=SMALL_WORKLOAD, small_dense=SMALL_DENSE_WORKLOAD, kimi_trace=TRACE_WORKLOAD, fp8_grid=FP8_WORKLOAD)[args.workload])
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -120,7 +120,7 @@ class DAMoE:
     """One context = one layer shape (k, E, H, I) with scratch for up to max_T tokens."""
 
     def __init__(self, max_T: int, k: int, E: int, H: int, I: int, dtype: int = BF16, device: int = 0):
-        self.max_T, self.k, self.E, self.H, self.I, self.device = max_T, k, E, H, I, device
+        self.max_T, self.k, self.E, self.H, self.I, self.device, self.dtype = max_T, k, E, H, I, device, dtype
         self._ctx = ctypes.c_void_p()
         rc = _lib.damoe_create(ctypes.byref(self._ctx), device, max_T, k, E, H, I, dtype)
         if rc != OK:
@@ -167,6 +167,11 @@ class DAMoE:
                                               _ptr(topk_weights_host), T, variant, _ptr(out_host),
                                               _stream_ptr(stream)))
         return out_host
+
+    def set_fp8_scales(self, x_scale, w13_scale, w2_scale):
+        """FP8 contexts: block scales read by the following fused_moe calls."""
+        self._keep_scales = (x_scale, w13_scale, w2_scale)
+        self._check(_lib.damoe_set_fp8_scales(self._ctx, _ptr(x_scale), _ptr(w13_scale), _ptr(w2_scale)))
 
     def load_tuning_table(self, blob: bytes):
         self._check(_lib.damoe_load_tuning_table(self._ctx, blob, len(blob)))

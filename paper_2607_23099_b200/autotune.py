@@ -70,8 +70,9 @@ def fit_cost(rows, ns):
     V = len(ns)
     out = dict(c_fix=[0] * V, c_byte=[0] * V, c_reload=[0] * V, c_flop=[0] * V)
     for v in range(V):
-        pts = [(r["active"], r["tiles"][v], r["us"][v]) for r in rows]
+        pts = [(r["active"], r["tiles"][v], r["us"][v]) for r in rows if r["us"][v] < 1e8]
         if not pts:
+            out["c_fix"][v] = 1 << 36
             continue
         A = np.array([[1.0, a, max(0, t - a)] for a, t, _ in pts])
         y = np.array([us * 1e6 for _, _, us in pts])
@@ -127,17 +128,23 @@ def time_call(fn, reps):
     return statistics.median(ts)
 
 
-def sweep(shape, buckets, alphas, seeds, reps, log_path, weight_seed=12345, device="cuda:0"):
+def sweep(shape, buckets, alphas, seeds, reps, log_path, weight_seed=12345, device="cuda:0", dtype=None):
+    dtype = d.BF16 if dtype is None else dtype
+    fp8 = dtype == d.FP8_E4M3_BLOCK128
     E, k, H, I = shape["E"], shape["k"], shape["H"], shape["I"]
     V, ns = d.variant_count(), d.tile_ns()
+    VA = 4 if fp8 else V                        # variants built for this dtype
     done = {}
     if log_path and os.path.exists(log_path):
         for line in open(log_path):
             r = json.loads(line)
             done[(r["T"], str(r["alpha"]), r["seed"])] = r
     W = di.MoEWeights(weight_seed, E, H, I)
-    w13, w2 = W.materialize(device)
-    m = d.DAMoE(max(buckets), k, E, H, I)
+    if fp8:
+        w13, w13s, w2, w2s = W.materialize_fp8(device)
+    else:
+        w13, w2 = W.materialize(device)
+    m = d.DAMoE(max(buckets), k, E, H, I, dtype=dtype)
     log = open(log_path, "a") if log_path else None
     result = {}
     for T in buckets:
@@ -155,11 +162,15 @@ def sweep(shape, buckets, alphas, seeds, reps, log_path, weight_seed=12345, devi
                     else:
                         ids, wts, _ = di.routing_batch(seed + int(round(alpha * 1000)), T, k, E, alpha)
                     x = di.activations(seed, T, H, device)
+                    if fp8:
+                        x, xs = di.quantize_e4m3_blocks(x, 1, 128)
+                        m.set_fp8_scales(xs, w13s, w2s)
                     ids_d, w_d = torch.from_numpy(ids).to(device), torch.from_numpy(wts).to(device)
                     out = torch.empty(T, H, dtype=torch.bfloat16, device=device)
-                    for v in range(V):                       # warm-up
+                    for v in range(VA):                      # warm-up
                         m.fused_moe(x, w13, w2, ids_d, w_d, v, out=out)
-                    us = [time_call(lambda v=v: m.fused_moe(x, w13, w2, ids_d, w_d, v, out=out), reps) for v in range(V)]
+                    us = [time_call(lambda v=v: m.fused_moe(x, w13, w2, ids_d, w_d, v, out=out), reps) for v in range(VA)]
+                    us += [1e9] * (V - VA)                   # variants not built for this dtype
                     meta = m.debug_fetch(T)
                     hist = np.bincount(ids.reshape(-1), minlength=E)
                     r = dict(T=T, alpha=alpha, seed=s, us=us, counts=hist.tolist(), active=int((hist > 0).sum()),
@@ -187,14 +198,16 @@ def main():
     ap.add_argument("--mode", default="exemplar", choices=["exemplar", "bins", "cost"])
     ap.add_argument("--out", required=True)
     ap.add_argument("--log", default=None)
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp8"])
     args = ap.parse_args()
+    dtype = d.BF16 if args.dtype == "bf16" else d.FP8_E4M3_BLOCK128
     shape = SHAPES[args.shape]
     buckets = [int(t) for t in args.buckets.split(",")]
     alphas = [float(a) for a in args.alphas.split(",")]
-    result, ns, V = sweep(shape, buckets, alphas, args.seeds, args.reps, args.log)
+    result, ns, V = sweep(shape, buckets, alphas, args.seeds, args.reps, args.log, dtype=dtype)
     table = dict(mode=dict(exemplar=d.MODE_EXEMPLAR, bins=d.MODE_EFFEXP_BINS, cost=d.MODE_COST)[args.mode],
                  buckets=[build_bucket(T, result[T], ns, V) for T in buckets])
-    blob = tuning.pack_table(table, shape["E"], shape["k"], shape["H"], shape["I"], d.BF16, V)
+    blob = tuning.pack_table(table, shape["E"], shape["k"], shape["H"], shape["I"], dtype, V)
     os.makedirs(os.path.dirname(os.path.abspath(args.out)), exist_ok=True)
     open(args.out, "wb").write(blob)
     # landscape report

@@ -39,7 +39,8 @@ struct damoe_ctx {
   const float* x_scale = nullptr;
   const float* w13_scale = nullptr;
   const float* w2_scale = nullptr;
-  int num_variants() const { return dtype == DAMOE_BF16 ? kNumVariants : kNumVariantsFp8; }
+  bool pairs_ok = false;  // CTA-pair variants need an even number of 128-row weight tiles in both GEMMs
+  int num_variants() const { return dtype != DAMOE_BF16 ? kNumVariantsFp8 : pairs_ok ? kNumVariants : kNumVariants1Cta; }
   // staging for the host-buffer entry point
   void *st_x = nullptr, *st_ids = nullptr, *st_w = nullptr, *st_out = nullptr;
   // stage timing
@@ -111,7 +112,7 @@ void default_cost_model(const damoe_ctx* c, int64_t* cost) {
   const double flops_col = 6.0 * c->H * c->I;
   for (int v = 0; v < kNumVariants; ++v) {
     const int n = variant_desc(v).tile_n;
-    const double eff = 0.75 * (n >= 128 ? 1.0 : n / 128.0);
+    const double eff = (variant_desc(v).cta_group == 2 ? 0.9 : 0.75) * (n >= 128 ? 1.0 : n / 128.0);
     cost[0 * kNumVariants + v] = 0;
     cost[1 * kNumVariants + v] = static_cast<int64_t>(wbytes / 6.5e12 * 1e12);
     cost[2 * kNumVariants + v] = static_cast<int64_t>(wbytes / 13e12 * 1e12);
@@ -215,6 +216,7 @@ int damoe_create(damoe_ctx** out, int device, int max_T, int k, int E, int H, in
   if (!c) return DAMOE_ERR_WORKSPACE;
   c->device = device; c->max_T = max_T; c->k = k; c->E = E; c->H = H; c->I = I; c->dtype = dtype;
   c->max_P = max_T * k;
+  c->pairs_ok = (I / 128) % 2 == 0 && (H / 128) % 2 == 0;
   auto bail = [&](int code) {
     damoe_destroy(c);
     return code;
@@ -224,7 +226,8 @@ int damoe_create(damoe_ctx** out, int device, int max_T, int k, int E, int H, in
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return bail(DAMOE_ERR_CUDA);
   if (prop.major != 10) return bail(DAMOE_ERR_UNSUPPORTED_SHAPE);  // tcgen05 kernels: sm_100a only
   c->sm_count = prop.multiProcessorCount;
-  if (gemm_configure() != cudaSuccess || gemm8_configure() != cudaSuccess) return bail(DAMOE_ERR_CUDA);
+  if (gemm_configure() != cudaSuccess || gemm8_configure() != cudaSuccess || gemm2cta_configure() != cudaSuccess)
+    return bail(DAMOE_ERR_CUDA);
 
   // one arena; 1024-byte aligned slices
   const size_t P = c->max_P;
@@ -512,17 +515,32 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
       DAMOE_CUDA(c, launch_gemm8(1, -1, false, m2, g2, c->sm_count, st));
     }
   } else if (known >= 0) {
-    DAMOE_CUDA(c, launch_gemm(0, known, false, m13, ga, c->sm_count, st));
-    DAMOE_MARK(3);
-    DAMOE_CUDA(c, launch_gemm(1, known, false, m2, ga, c->sm_count, st));
+    if (known >= kNumVariants1Cta) {
+      DAMOE_CUDA(c, launch_gemm2cta(0, known, false, m13, ga, c->sm_count, st));
+      DAMOE_MARK(3);
+      DAMOE_CUDA(c, launch_gemm2cta(1, known, false, m2, ga, c->sm_count, st));
+    } else {
+      DAMOE_CUDA(c, launch_gemm(0, known, false, m13, ga, c->sm_count, st));
+      DAMOE_MARK(3);
+      DAMOE_CUDA(c, launch_gemm(1, known, false, m2, ga, c->sm_count, st));
+    }
   } else if (c->dispatch == DAMOE_DISPATCH_PREDICATED) {
-    for (int v = 0; v < kNumVariants; ++v) DAMOE_CUDA(c, launch_gemm(0, v, true, m13, ga, c->sm_count, st));
+    const int nv = c->num_variants();
+    for (int v = 0; v < nv; ++v)
+      DAMOE_CUDA(c, v < kNumVariants1Cta ? launch_gemm(0, v, true, m13, ga, c->sm_count, st)
+                                         : launch_gemm2cta(0, v, true, m13, ga, c->sm_count, st));
     DAMOE_MARK(3);
-    for (int v = 0; v < kNumVariants; ++v) DAMOE_CUDA(c, launch_gemm(1, v, true, m2, ga, c->sm_count, st));
+    for (int v = 0; v < nv; ++v)
+      DAMOE_CUDA(c, v < kNumVariants1Cta ? launch_gemm(1, v, true, m2, ga, c->sm_count, st)
+                                         : launch_gemm2cta(1, v, true, m2, ga, c->sm_count, st));
   } else {
+    // one branching kernel for the 1-CTA variants, one (cluster launch) for the CTA-pair variants;
+    // the one that does not hold the chosen variant exits at once
     DAMOE_CUDA(c, launch_gemm(0, -1, false, m13, ga, c->sm_count, st));
+    if (c->pairs_ok) DAMOE_CUDA(c, launch_gemm2cta(0, -2, false, m13, ga, c->sm_count, st));
     DAMOE_MARK(3);
     DAMOE_CUDA(c, launch_gemm(1, -1, false, m2, ga, c->sm_count, st));
+    if (c->pairs_ok) DAMOE_CUDA(c, launch_gemm2cta(1, -2, false, m2, ga, c->sm_count, st));
   }
   DAMOE_MARK(4);
   DAMOE_CUDA(c, launch_reduce(c->ws, static_cast<__nv_bfloat16*>(out), T, c->k, c->H, st));

@@ -24,10 +24,12 @@ struct VariantDesc {
   int stages13;   // pipeline depth of the gate/up GEMM
   int stages2;    // pipeline depth of the down GEMM
 };
-constexpr int kNumVariants = 5;
+constexpr int kNumVariants = 7;
+constexpr int kNumVariants1Cta = 5;  // ids 0..4: one CTA per tile; ids 5..6: CTA pairs (cta_group::2, M = 256)
 __host__ __device__ constexpr VariantDesc variant_desc(int v) {
   constexpr VariantDesc t[kNumVariants] = {
-      {16, 128, 1, 6, 10}, {32, 128, 1, 5, 10}, {64, 128, 1, 5, 8}, {128, 128, 1, 4, 6}, {256, 128, 1, 3, 4}};
+      {16, 128, 1, 6, 10}, {32, 128, 1, 5, 10}, {64, 128, 1, 5, 8}, {128, 128, 1, 4, 6}, {256, 128, 1, 3, 4},
+      {128, 256, 2, 5, 8}, {256, 256, 2, 4, 6}};
   return t[v];
 }
 
@@ -99,6 +101,11 @@ struct GemmArgs {
 cudaError_t launch_gemm(int kind, int variant, bool predicated, const GemmMaps& maps, const GemmArgs& args,
                         int sm_count, cudaStream_t stream);
 cudaError_t gemm_configure();  // opt-in shared-memory sizes, once per device
+// gemm_2cta.cu: variants 5..6 (CTA pairs).  variant == -2: one kernel that branches between them
+// and exits at once when *variant_id names a 1-CTA variant.
+cudaError_t launch_gemm2cta(int kind, int variant, bool predicated, const GemmMaps& maps, const GemmArgs& args,
+                            int sm_count, cudaStream_t stream);
+cudaError_t gemm2cta_configure();
 
 // gemm_fp8.cu: the same family on kind::f8f6f4 with per-128-K-block scale promotion.
 constexpr int kNumVariantsFp8 = 4;  // N = 16, 32, 64, 128 (variant ids 0..3)

@@ -1,0 +1,348 @@
+// Grouped expert GEMMs with CTA pairs (tcgen05 cta_group::2) for the compute-bound regime.
+//
+// Two CTAs of a cluster work on one item: (expert, PAIR of adjacent 128-row weight tiles,
+// token tile of width N_v).  The MMA has M = 256: CTA rank r supplies weight rows
+// [m0 + 128 r, m0 + 128 r + 128) and keeps their accumulator rows in its own TMEM, and each
+// CTA stages only HALF of the token tile (N_v / 2 rows); the tensor core reads both halves.
+// Per MAC this halves the L2 -> shared-memory operand traffic of the 1-CTA kernel, which is
+// what bounds it once the experts receive hundreds of tokens.
+//
+// Roles per CTA (6 warps): warp 0 TMA producer (its own weight tiles and its half of the
+// tokens; the transaction bytes of both CTAs complete on the leader's "full" barrier), warp 1
+// TMEM allocation, and on the leader (rank 0) the single MMA-issuing thread for the pair;
+// warps 2..5 epilogue on the CTA's own TMEM.  tcgen05.commit multicasts the "stage empty" and
+// "accumulator full" arrivals to both CTAs; the epilogue warps of both CTAs arrive on the
+// leader's "accumulator empty" barrier.  No TMA multicast is used.
+//
+// Every mbarrier wait is bounded; the only unbounded synchronisation is the cluster barrier at
+// start-up and at teardown, which both CTAs always reach.
+#include "common.cuh"
+#include "gemm_common.cuh"
+#include "ptx.cuh"
+
+namespace damoe {
+
+namespace {
+
+constexpr int kThreads2 = 192;
+constexpr int kABytes2 = kTileM * kBK * 2;
+constexpr int kTailBytes2 = 2 * (kMaxE + 1) * 4 + 512;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const void* tmap, uint32_t leader_bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], "
+      "[%2];" ::"r"(dst),
+      "l"(tmap), "r"(leader_bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_result, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs
+// issued so far have completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+      "h"(mask)
+      : "memory");
+}
+
+template <int KIND, int BN, int STAGES>
+struct Cfg2 {
+  static constexpr int kATiles = (KIND == 0) ? 2 : 1;
+  static constexpr int kBRows = BN / 2;                 // token rows staged by each CTA
+  static constexpr int kBBytes = kBRows * kBK * 2;
+  static constexpr int kStageBytes = kATiles * kABytes2 + kBBytes;
+  static constexpr int kAccCols = kATiles * BN;
+  static constexpr int kNumAcc = (2 * kAccCols <= 512) ? 2 : 1;
+  static constexpr int kTmemCols = (kNumAcc * kAccCols <= 256) ? 256 : 512;
+  static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + kTailBytes2;
+  static_assert(kStageBytes % 1024 == 0, "operand tiles must stay 1024-byte aligned for the 128B swizzle");
+  static_assert(kSmemBytes <= 232448, "over the 227 KB shared-memory limit");
+};
+
+template <int KIND, int BN, int STAGES>
+__device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUtensorMap* tmap_act, const GemmArgs& a,
+                                           int variant, uint8_t* smem_raw) {
+  using C = Cfg2<KIND, BN, STAGES>;
+  const int K = (KIND == 0) ? a.H : a.I;
+  const int MROWS = (KIND == 0) ? 2 * a.I : a.H;
+  const int MT2 = ((KIND == 0) ? a.I : a.H) / (2 * kTileM);  // weight-tile PAIRS per expert
+  const int KB = K / kBK;
+  const int E = a.E;
+  const uint32_t rank = cluster_ctarank();
+  const int cluster_id = blockIdx.x >> 1;
+  const int num_clusters = gridDim.x >> 1;
+
+  const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* tail = smem_raw + (tiles_base - smem_u32(smem_raw)) + STAGES * C::kStageBytes;
+  int* s_pref = reinterpret_cast<int*>(tail);
+  int* s_off = s_pref + (kMaxE + 1);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_off + (kMaxE + 1));
+  const uint32_t bar_full = smem_u32(bars);             // used on the leader only
+  const uint32_t bar_empty = bar_full + 8u * STAGES;    // one set per CTA, fed by multicast commits
+  const uint32_t bar_tfull = bar_empty + 8u * STAGES;   // one set per CTA, fed by multicast commits
+  const uint32_t bar_tempty = bar_tfull + 16u;          // used on the leader only: 8 epilogue warps arrive
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  const int32_t* pref_g = a.ntile_prefix + variant * (E + 1);
+  for (int i = tid; i <= E; i += kThreads2) {
+    s_pref[i] = pref_g[i];
+    s_off[i] = a.offsets[i];
+  }
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_empty + 8u * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_tfull + 8u * b, 1);
+      mbar_init(bar_tempty + 8u * b, 8);
+    }
+    *s_abort = 0;
+    fence_mbar_init();
+    fence_proxy_async_smem();
+    prefetch_tensormap(tmap_w);
+    prefetch_tensormap(tmap_act);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(s_tmem), C::kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // barriers of both CTAs are initialised before anyone signals them
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  const int total = s_pref[E] * MT2;
+
+  if (warp == 0) {
+    // ---------------- TMA producer (both CTAs) ----------------
+    if (lane == 0) {
+      int it = 0;
+      bool ok = true;
+      for (int w = cluster_id; ok && w < total; w += num_clusters) {
+        const Item item = decode_item(w, s_pref, s_off, E, MT2, BN);   // item.m_tile = pair index
+        const int n_eff = (item.valid + 15) & ~15;
+        const int n_use = n_eff < BN ? n_eff : BN;
+        const int row_a = item.e * MROWS + (2 * item.m_tile + static_cast<int>(rank)) * kTileM;
+        const int row_b = item.q0 + static_cast<int>(rank) * (n_use >> 1);  // this CTA's half of the token columns
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, s_abort)) {
+            ok = false;
+            break;
+          }
+          const uint32_t full_leader = map_to_cta(bar_full + 8u * s, 0);
+          const uint32_t sa = tiles_base + s * C::kStageBytes;
+          if (rank == 0) mbar_arrive_expect_tx(bar_full + 8u * s, 2u * C::kStageBytes);  // both CTAs' bytes
+          tma_load_2d_pair(sa, tmap_w, full_leader, kb * kBK, row_a);
+          if (KIND == 0) tma_load_2d_pair(sa + kABytes2, tmap_w, full_leader, kb * kBK, row_a + a.I);
+          tma_load_2d_pair(sa + C::kATiles * kABytes2, tmap_act, full_leader, kb * kBK, row_b);
+        }
+      }
+      (void)ok;
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (leader CTA only) ----------------
+    if (lane == 0 && rank == 0) {
+      int it = 0, tile_i = 0;
+      bool ok = true;
+      for (int w = cluster_id; ok && w < total; w += num_clusters, ++tile_i) {
+        const Item item = decode_item(w, s_pref, s_off, E, MT2, BN);
+        const int n_eff = (item.valid + 15) & ~15;
+        const uint32_t idesc = umma_idesc_bf16(2 * kTileM, n_eff < BN ? n_eff : BN);
+        const int buf = tile_i % C::kNumAcc;
+        const uint32_t aph = (tile_i / C::kNumAcc) & 1;
+        if (!mbar_wait(bar_tempty + 8u * buf, aph ^ 1u, s_abort)) break;
+        tc_fence_after();
+        const uint32_t d0 = tmem_base + buf * C::kAccCols;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(bar_full + 8u * s, ph, s_abort)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t sa = tiles_base + s * C::kStageBytes;
+          const uint64_t da0 = umma_desc_sw128(sa);
+          const uint64_t da1 = umma_desc_sw128(sa + kABytes2);
+          const uint64_t db = umma_desc_sw128(sa + C::kATiles * kABytes2);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) {
+            const uint32_t acc = (kb | k) ? 1u : 0u;
+            umma_bf16_pair(d0, da0 + 2u * k, db + 2u * k, idesc, acc);
+            if (KIND == 0) umma_bf16_pair(d0 + BN, da1 + 2u * k, db + 2u * k, idesc, acc);
+          }
+          umma_commit_pair(bar_empty + 8u * s);
+        }
+        if (ok) umma_commit_pair(bar_tfull + 8u * buf);
+      }
+    }
+  } else {
+    // ---------------- epilogue (both CTAs, each on its own 128 accumulator rows) ----------------
+    const uint32_t lane_base = (warp & 3) * 32;
+    int tile_i = 0;
+    for (int w = cluster_id; w < total; w += num_clusters, ++tile_i) {
+      const Item item = decode_item(w, s_pref, s_off, E, MT2, BN);
+      const int buf = tile_i % C::kNumAcc;
+      const uint32_t aph = (tile_i / C::kNumAcc) & 1;
+      if (!mbar_wait(bar_tfull + 8u * buf, aph, s_abort)) break;
+      tc_fence_after();
+      const int ch = (2 * item.m_tile + static_cast<int>(rank)) * kTileM + lane_base + lane;
+      const uint32_t t0 = tmem_base + (lane_base << 16) + buf * C::kAccCols;
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 16) {
+        if (c0 >= item.valid) break;
+        uint32_t g[16], u[16];
+        tmem_ld_x16(t0 + c0, g);
+        if (KIND == 0) tmem_ld_x16(t0 + BN + c0, u);
+        tmem_ld_wait();
+        if (KIND == 0) {
+          __nv_bfloat16* dst = a.h + static_cast<size_t>(item.q0 + c0) * a.I + ch;
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c0 + j < item.valid)
+              dst[static_cast<size_t>(j) * a.I] = __float2bfloat16_rn(silu_mul(__uint_as_float(g[j]), __uint_as_float(u[j])));
+        } else {
+          float* dst = a.y + static_cast<size_t>(item.q0 + c0) * a.H + ch;
+          const float* wq = a.w_sorted + item.q0 + c0;
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c0 + j < item.valid) dst[static_cast<size_t>(j) * a.H] = __ldg(wq + j) * __uint_as_float(g[j]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_tempty + 8u * buf, 0));
+    }
+  }
+
+  // ---------------- teardown ----------------
+  if (*s_abort) {  // give copies that are still in flight time to land before the shared memory is released
+    const uint64_t t_end = global_timer_ns() + 2000000ull;
+    while (global_timer_ns() < t_end) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the leader's MMAs read the peer's shared memory until here
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc_pair(tmem_base, C::kTmemCols);
+  }
+  if (tid == 0 && *s_abort) atomicOr(a.status, DAMOE_STATUS_WAIT_TIMEOUT);
+}
+
+template <int KIND, int V>
+struct VCfg2 {
+  static constexpr int kBN = variant_desc(V).tile_n;
+  static constexpr int kStages = (KIND == 0) ? variant_desc(V).stages13 : variant_desc(V).stages2;
+  using C = Cfg2<KIND, kBN, kStages>;
+};
+
+template <int KIND, int V>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
+    gemm2_fixed_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_act,
+                       const GemmArgs a, const int predicated) {
+  extern __shared__ uint8_t smem_raw[];
+  if (predicated && *a.variant_id != V) return;
+  gemm2_body<KIND, VCfg2<KIND, V>::kBN, VCfg2<KIND, V>::kStages>(&tmap_w, &tmap_act, a, V, smem_raw);
+}
+
+template <int KIND>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
+    gemm2_branch_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  const int v = *a.variant_id;
+  if (v == 5) gemm2_body<KIND, VCfg2<KIND, 5>::kBN, VCfg2<KIND, 5>::kStages>(&maps.w, &maps.act[2], a, 5, smem_raw);
+  else if (v == 6) gemm2_body<KIND, VCfg2<KIND, 6>::kBN, VCfg2<KIND, 6>::kStages>(&maps.w, &maps.act[3], a, 6, smem_raw);
+}
+
+template <int KIND>
+constexpr int max_smem2() {
+  return VCfg2<KIND, 5>::C::kSmemBytes > VCfg2<KIND, 6>::C::kSmemBytes ? VCfg2<KIND, 5>::C::kSmemBytes
+                                                                       : VCfg2<KIND, 6>::C::kSmemBytes;
+}
+
+template <int KIND, int V>
+cudaError_t launch_fixed2(const GemmMaps& maps, const GemmArgs& args, bool predicated, int grid, cudaStream_t st) {
+  constexpr int kHalfRowsVariant = (VCfg2<KIND, V>::kBN == 128) ? 2 : 3;  // tensor map whose box has N_v / 2 rows
+  gemm2_fixed_kernel<KIND, V><<<grid & ~1, kThreads2, VCfg2<KIND, V>::C::kSmemBytes, st>>>(
+      maps.w, maps.act[kHalfRowsVariant], args, predicated ? 1 : 0);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t gemm2cta_configure() {
+  cudaError_t e;
+#define DAMOE_CFG2(K, V)                                                                                   \
+  if ((e = cudaFuncSetAttribute(gemm2_fixed_kernel<K, V>, cudaFuncAttributeMaxDynamicSharedMemorySize,     \
+                                VCfg2<K, V>::C::kSmemBytes)) != cudaSuccess)                               \
+    return e;
+  DAMOE_CFG2(0, 5) DAMOE_CFG2(0, 6) DAMOE_CFG2(1, 5) DAMOE_CFG2(1, 6)
+#undef DAMOE_CFG2
+  if ((e = cudaFuncSetAttribute(gemm2_branch_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem2<0>())) !=
+      cudaSuccess)
+    return e;
+  return cudaFuncSetAttribute(gemm2_branch_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem2<1>());
+}
+
+cudaError_t launch_gemm2cta(int kind, int variant, bool predicated, const GemmMaps& maps, const GemmArgs& args,
+                            int sm_count, cudaStream_t stream) {
+  if (variant == -2) {
+    if (kind == 0) gemm2_branch_kernel<0><<<sm_count & ~1, kThreads2, max_smem2<0>(), stream>>>(maps, args);
+    else gemm2_branch_kernel<1><<<sm_count & ~1, kThreads2, max_smem2<1>(), stream>>>(maps, args);
+    return cudaGetLastError();
+  }
+  if (kind == 0) {
+    if (variant == 5) return launch_fixed2<0, 5>(maps, args, predicated, sm_count, stream);
+    if (variant == 6) return launch_fixed2<0, 6>(maps, args, predicated, sm_count, stream);
+  } else {
+    if (variant == 5) return launch_fixed2<1, 5>(maps, args, predicated, sm_count, stream);
+    if (variant == 6) return launch_fixed2<1, 6>(maps, args, predicated, sm_count, stream);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace damoe

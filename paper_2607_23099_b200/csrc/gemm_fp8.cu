@@ -54,7 +54,8 @@ struct Cfg8 {
   static constexpr int kBBytes = BN * kBK8;
   static constexpr int kStageBytes = kATiles * kABytes8 + kBBytes;
   static constexpr int kAccCols = kATiles * BN;   // one partial buffer
-  static constexpr int kTmemColsRaw = 2 * kAccCols;
+  static constexpr int kNumPartials = (4 * kAccCols <= 512) ? 4 : 2;  // partial buffers in flight
+  static constexpr int kTmemColsRaw = kNumPartials * kAccCols;
   static constexpr int kTmemCols = kTmemColsRaw <= 32 ? 32 : kTmemColsRaw <= 64 ? 64 : kTmemColsRaw <= 128 ? 128
                                    : kTmemColsRaw <= 256 ? 256 : 512;
   static constexpr int kCW = BN / 2;              // token columns per epilogue warp
@@ -103,9 +104,10 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
   const uint32_t bar_full = smem_u32(bars);
   const uint32_t bar_empty = bar_full + 8u * STAGES;
   const uint32_t bar_pfull = bar_empty + 8u * STAGES;
-  const uint32_t bar_pempty = bar_pfull + 16u;
-  const uint32_t bar_xchg = bar_pempty + 16u;  // one per column half: the 4 warps sharing it exchange amax
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 6);
+  const uint32_t bar_pempty = bar_pfull + 32u;
+  const uint32_t bar_xchg = bar_pempty + 32u;  // one per column half: the 4 warps sharing it exchange amax
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 10);
+  constexpr int NP = C::kNumPartials;
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   float* s_amax = reinterpret_cast<float*>(s_tmem + 2);  // [2 buffers][4 quadrants][BN]
 
@@ -121,11 +123,11 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
       mbar_init(bar_full + 8u * s, 1);
       mbar_init(bar_empty + 8u * s, 1);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < 4; ++b) {
       mbar_init(bar_pfull + 8u * b, 1);
       mbar_init(bar_pempty + 8u * b, 8);
-      mbar_init(bar_xchg + 8u * b, 4);
     }
+    for (int b = 0; b < 2; ++b) mbar_init(bar_xchg + 8u * b, 4);
     *s_abort = 0;
     fence_mbar_init();
     fence_proxy_async_smem();
@@ -183,8 +185,8 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
-          const int pb = it & 1;
-          const uint32_t pph = (it >> 1) & 1;
+          const int pb = it % NP;
+          const uint32_t pph = (it / NP) & 1;
           if (!mbar_wait(bar_pempty + 8u * pb, pph ^ 1u, s_abort) || !mbar_wait(bar_full + 8u * s, ph, s_abort)) {
             ok = false;
             break;
@@ -230,8 +232,8 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
       }
       bool ok = true;
       for (int kb = 0; kb < KB; ++kb, ++it) {
-        const int pb = it & 1;
-        const uint32_t pph = (it >> 1) & 1;
+        const int pb = it % NP;
+        const uint32_t pph = (it / NP) & 1;
         // this lane's share of the activation scales of the K block: lane l holds column col0+l (and +32)
         const float* xs = a.act_scale_T + static_cast<size_t>(kb) * a.max_P + item.q0 + col0;
         float sx0 = 0.f, sx1 = 0.f;

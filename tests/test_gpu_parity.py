@@ -166,7 +166,7 @@ def _table_for(E, k, T_buckets, mode, V, ns):
 
 def test_selected_variant_matches_oracle_given_the_same_table(d):
     from paper_2607_23099_b200 import tuning
-    E, k, H, I = 64, 4, 256, 128
+    E, k, H, I = 64, 4, 256, 256          # even numbers of 128-row weight tiles: CTA-pair variants exist too
     V, ns = d.variant_count(), d.tile_ns()
     W = di.MoEWeights(1, E, H, I)
     w13, w2 = W.materialize("cuda")
