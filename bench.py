@@ -315,9 +315,10 @@ def run_ours(args):
     cells = make_cells(device)
     m = d.DAMoE(w["T"], w["k"], w["E"], w["H"], w["I"], dtype=d.FP8_E4M3_BLOCK128 if fp8 else d.BF16, device=local)
     table = "built-in cost model"
-    if os.path.exists(table_path(w)) and not args.no_table:
-        m.load_tuning_table(open(table_path(w), "rb").read())
-        table = os.path.relpath(table_path(w), ROOT)
+    tpath = args.table or table_path(w)
+    if os.path.exists(tpath) and not args.no_table:
+        m.load_tuning_table(open(tpath, "rb").read())
+        table = os.path.relpath(tpath, ROOT)
     out = torch.empty(w["T"], w["H"], dtype=torch.bfloat16, device=device)
     out_host = torch.empty(w["T"], w["H"], dtype=torch.bfloat16).pin_memory()
     stream = torch.cuda.current_stream()
@@ -450,6 +451,7 @@ def main():
     ap.add_argument("--workload", default="headline", choices=["headline", "small", "small_dense", "kimi_trace", "fp8_grid"],
                     help="'small' is the reduced case used for ncu captures; 'kimi_trace' the 500-batch serving-trace stand-in")
     ap.add_argument("--no-table", action="store_true", help="ignore the committed tuning table")
+    ap.add_argument("--table", default=None, help="tuning table file to load instead of the committed one")
     ap.add_argument("--variant", type=int, default=None, help="force this kernel variant in the timed steps (profiling)")
     args = ap.parse_args()
     if args.workload != "headline":

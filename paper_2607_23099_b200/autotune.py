@@ -85,15 +85,24 @@ def fit_cost(rows, ns):
     return out
 
 
-def build_bucket(T, cells, ns, V):
-    """cells: list of dict(alpha, counts[S][E], us[S][V], active[S], tiles[S][V])."""
+def build_bucket(T, cells, ns, V, margin=0.02):
+    """cells: list of dict(alpha, counts[S][E], us[S][V], active[S], tiles[S][V]).
+
+    A distribution is paired with its fastest variant only when that variant beats the
+    bucket's static choice by more than ``margin`` (timing noise between near-equal variants
+    must not move the dispatcher off the static choice for nothing)."""
     ex, exv, rows, effs = [], [], [], []
     static_variant = 2
     for c in cells:
+        if c["alpha"] == UNIFORM:
+            static_variant = int(np.argmin(np.mean(np.array(c["us"]), axis=0)))
+    for c in cells:
         mean_us = np.mean(np.array(c["us"]), axis=0)
         best = int(np.argmin(mean_us))
+        if mean_us[static_variant] <= mean_us[best] * (1.0 + margin):
+            best = static_variant
         if c["alpha"] == UNIFORM:
-            static_variant = best
+            pass
         else:
             ex.append(exemplar_q30(c["counts"]))
             exv.append(best)
@@ -126,6 +135,26 @@ def time_call(fn, reps):
         b.synchronize()
         ts.append(a.elapsed_time(b) * 1e3)
     return statistics.median(ts)
+
+
+def cells_from_log(log_path, buckets, alphas, seeds):
+    """Rebuilds the sweep result from its log alone (no GPU)."""
+    done = {}
+    for line in open(log_path):
+        r = json.loads(line)
+        done[(r["T"], str(r["alpha"]), r["seed"])] = r
+    result = {}
+    for T in buckets:
+        cells = []
+        for alpha in list(alphas) + [UNIFORM]:
+            cell = dict(alpha=alpha, counts=[], us=[], active=[], tiles=[])
+            for s in range(seeds):
+                r = done[(T, str(alpha), s)]
+                for key in ("counts", "us", "active", "tiles"):
+                    cell[key].append(r[key])
+            cells.append(cell)
+        result[T] = cells
+    return result
 
 
 def sweep(shape, buckets, alphas, seeds, reps, log_path, weight_seed=12345, device="cuda:0", dtype=None):
@@ -199,17 +228,25 @@ def main():
     ap.add_argument("--out", required=True)
     ap.add_argument("--log", default=None)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp8"])
+    ap.add_argument("--from-log", action="store_true", help="build the table from --log alone, without a GPU")
+    ap.add_argument("--margin", type=float, default=0.02, help="minimum gain over the static choice to leave it")
     args = ap.parse_args()
     dtype = d.BF16 if args.dtype == "bf16" else d.FP8_E4M3_BLOCK128
     shape = SHAPES[args.shape]
     buckets = [int(t) for t in args.buckets.split(",")]
     alphas = [float(a) for a in args.alphas.split(",")]
-    result, ns, V = sweep(shape, buckets, alphas, args.seeds, args.reps, args.log, dtype=dtype)
-    table = dict(mode=dict(exemplar=d.MODE_EXEMPLAR, bins=d.MODE_EFFEXP_BINS, cost=d.MODE_COST)[args.mode],
-                 buckets=[build_bucket(T, result[T], ns, V) for T in buckets])
-    blob = tuning.pack_table(table, shape["E"], shape["k"], shape["H"], shape["I"], dtype, V)
+    if args.from_log:
+        result, ns, V = cells_from_log(args.log, buckets, alphas, args.seeds), d.tile_ns(), d.variant_count()
+    else:
+        result, ns, V = sweep(shape, buckets, alphas, args.seeds, args.reps, args.log, dtype=dtype)
+    modes = dict(exemplar=d.MODE_EXEMPLAR, bins=d.MODE_EFFEXP_BINS, cost=d.MODE_COST)
+    bucket_rows = [build_bucket(T, result[T], ns, V, margin=args.margin) for T in buckets]
     os.makedirs(os.path.dirname(os.path.abspath(args.out)), exist_ok=True)
-    open(args.out, "wb").write(blob)
+    for name, mode in modes.items():
+        # the requested mode goes to --out; the other two land beside it for comparison
+        path = args.out if name == args.mode else args.out + "." + name
+        blob = tuning.pack_table(dict(mode=mode, buckets=bucket_rows), shape["E"], shape["k"], shape["H"], shape["I"], dtype, V)
+        open(path, "wb").write(blob)
     # landscape report
     print(f"# variants N = {ns}; microseconds per layer, mean over {args.seeds} seeds; * = best")
     for T in buckets:

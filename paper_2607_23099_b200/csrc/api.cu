@@ -534,13 +534,13 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
       DAMOE_CUDA(c, v < kNumVariants1Cta ? launch_gemm(1, v, true, m2, ga, c->sm_count, st)
                                          : launch_gemm2cta(1, v, true, m2, ga, c->sm_count, st));
   } else {
-    // one branching kernel for the 1-CTA variants, one (cluster launch) for the CTA-pair variants;
-    // the one that does not hold the chosen variant exits at once
-    DAMOE_CUDA(c, launch_gemm(0, -1, false, m13, ga, c->sm_count, st));
+    // one persistent kernel per GEMM that branches on the variant id; when the CTA-pair variants
+    // exist it is launched as clusters of two so that it can hold the whole family
     if (c->pairs_ok) DAMOE_CUDA(c, launch_gemm2cta(0, -2, false, m13, ga, c->sm_count, st));
+    else DAMOE_CUDA(c, launch_gemm(0, -1, false, m13, ga, c->sm_count, st));
     DAMOE_MARK(3);
-    DAMOE_CUDA(c, launch_gemm(1, -1, false, m2, ga, c->sm_count, st));
     if (c->pairs_ok) DAMOE_CUDA(c, launch_gemm2cta(1, -2, false, m2, ga, c->sm_count, st));
+    else DAMOE_CUDA(c, launch_gemm(1, -1, false, m2, ga, c->sm_count, st));
   }
   DAMOE_MARK(4);
   DAMOE_CUDA(c, launch_reduce(c->ws, static_cast<__nv_bfloat16*>(out), T, c->k, c->H, st));

@@ -1,0 +1,211 @@
+// The 1-CTA grouped GEMM body (tcgen05 cta_group::1), shared by the fixed-variant kernels and by
+// the branching kernels.  See gemm.cu for the description of the kernel.
+#pragma once
+#include "common.cuh"
+#include "gemm_common.cuh"
+#include "ptx.cuh"
+
+namespace damoe {
+namespace {
+
+constexpr int kGemmThreads = 192;
+constexpr int kABytes = kTileM * kBK * 2;  // one 128 x 64 bf16 weight tile
+constexpr int kTailBytes = 2 * (kMaxE + 1) * 4 + 512;  // prefix + offsets copies, barriers, flags
+
+template <int KIND, int BN, int STAGES>
+struct Cfg {
+  static constexpr int kATiles = (KIND == 0) ? 2 : 1;
+  static constexpr int kBBytes = BN * kBK * 2;
+  static constexpr int kStageBytes = kATiles * kABytes + kBBytes;
+  static constexpr int kAccCols = kATiles * BN;
+  static constexpr int kNumAcc = (2 * kAccCols <= 512) ? 2 : 1;
+  static constexpr int kTmemCols = (kNumAcc * kAccCols <= 32)    ? 32
+                                   : (kNumAcc * kAccCols <= 64)  ? 64
+                                   : (kNumAcc * kAccCols <= 128) ? 128
+                                   : (kNumAcc * kAccCols <= 256) ? 256
+                                                                 : 512;
+  static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + kTailBytes;
+  static_assert(kStageBytes % 1024 == 0, "operand tiles must stay 1024-byte aligned for the 128B swizzle");
+  static_assert(kSmemBytes <= 232448, "over the 227 KB shared-memory limit");
+};
+
+template <int KIND, int BN, int STAGES>
+__device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUtensorMap* tmap_act, const GemmArgs& a,
+                                          int variant, uint8_t* smem_raw) {
+  using C = Cfg<KIND, BN, STAGES>;
+  const int K = (KIND == 0) ? a.H : a.I;
+  const int MROWS = (KIND == 0) ? 2 * a.I : a.H;  // weight rows per expert in the [E*rows, K] view
+  const int MT = ((KIND == 0) ? a.I : a.H) / kTileM;
+  const int KB = K / kBK;
+  const int E = a.E;
+
+  const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* tail = smem_raw + (tiles_base - smem_u32(smem_raw)) + STAGES * C::kStageBytes;
+  int* s_pref = reinterpret_cast<int*>(tail);
+  int* s_off = s_pref + (kMaxE + 1);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_off + (kMaxE + 1));  // 8-byte aligned: tail offset is a multiple of 8
+  const uint32_t bar_full = smem_u32(bars);
+  const uint32_t bar_empty = bar_full + 8u * STAGES;
+  const uint32_t bar_tfull = bar_empty + 8u * STAGES;
+  const uint32_t bar_tempty = bar_tfull + 16u;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  const int32_t* pref_g = a.ntile_prefix + variant * (E + 1);
+  for (int i = tid; i <= E; i += kGemmThreads) {
+    s_pref[i] = pref_g[i];
+    s_off[i] = a.offsets[i];
+  }
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_empty + 8u * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_tfull + 8u * b, 1);
+      mbar_init(bar_tempty + 8u * b, 4);
+    }
+    *s_abort = 0;
+    fence_mbar_init();
+    fence_proxy_async_smem();
+    prefetch_tensormap(tmap_w);
+    prefetch_tensormap(tmap_act);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(s_tmem), C::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  const int total = s_pref[E] * MT;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int it = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
+        const Item item = decode_item(w, s_pref, s_off, E, MT, BN);
+        const int row_a = item.e * MROWS + item.m_tile * kTileM;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, s_abort)) {
+            ok = false;
+            break;
+          }
+          const uint32_t full = bar_full + 8u * s;
+          const uint32_t sa = tiles_base + s * C::kStageBytes;
+          mbar_arrive_expect_tx(full, C::kStageBytes);
+          tma_load_2d(sa, tmap_w, full, kb * kBK, row_a);
+          if (KIND == 0) tma_load_2d(sa + kABytes, tmap_w, full, kb * kBK, row_a + a.I);
+          tma_load_2d(sa + C::kATiles * kABytes, tmap_act, full, kb * kBK, item.q0);
+        }
+      }
+      if (!ok) {  // drain what is still in flight so no copy lands after the CTA has gone
+        int dummy = 0;
+        for (int j = (it > STAGES ? it - STAGES : 0); j < it; ++j)
+          mbar_wait(bar_full + 8u * (j % STAGES), (j / STAGES) & 1, &dummy, 200000000ull);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      int it = 0, tile_i = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; ok && w < total; w += gridDim.x, ++tile_i) {
+        // A ragged last token tile issues narrower MMAs: N is a field of the instruction
+        // descriptor, so only ceil16(valid) token columns cost tensor time.
+        const Item item = decode_item(w, s_pref, s_off, E, MT, BN);
+        const int n_eff = (item.valid + 15) & ~15;
+        const uint32_t idesc = umma_idesc_bf16(kTileM, n_eff < BN ? n_eff : BN);
+        const int buf = tile_i % C::kNumAcc;
+        const uint32_t aph = (tile_i / C::kNumAcc) & 1;
+        if (!mbar_wait(bar_tempty + 8u * buf, aph ^ 1u, s_abort)) break;
+        tc_fence_after();
+        const uint32_t d0 = tmem_base + buf * C::kAccCols;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(bar_full + 8u * s, ph, s_abort)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t sa = tiles_base + s * C::kStageBytes;
+          const uint64_t da0 = umma_desc_sw128(sa);
+          const uint64_t da1 = umma_desc_sw128(sa + kABytes);
+          const uint64_t db = umma_desc_sw128(sa + C::kATiles * kABytes);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) {
+            const uint32_t acc = (kb | k) ? 1u : 0u;
+            umma_bf16(d0, da0 + 2u * k, db + 2u * k, idesc, acc);  // +32 bytes per K=16 step
+            if (KIND == 0) umma_bf16(d0 + BN, da1 + 2u * k, db + 2u * k, idesc, acc);
+          }
+          umma_commit(bar_empty + 8u * s);  // stage is free once these MMAs have read it
+        }
+        if (ok) umma_commit(bar_tfull + 8u * buf);
+      }
+    }
+  } else {
+    // ---------------- epilogue ----------------
+    const uint32_t lane_base = (warp & 3) * 32;  // the TMEM lane quadrant this warp may read
+    int tile_i = 0;
+    for (int w = blockIdx.x; w < total; w += gridDim.x, ++tile_i) {
+      const Item item = decode_item(w, s_pref, s_off, E, MT, BN);
+      const int buf = tile_i % C::kNumAcc;
+      const uint32_t aph = (tile_i / C::kNumAcc) & 1;
+      if (!mbar_wait(bar_tfull + 8u * buf, aph, s_abort)) break;
+      tc_fence_after();
+      const int ch = item.m_tile * kTileM + lane_base + lane;
+      const uint32_t t0 = tmem_base + (lane_base << 16) + buf * C::kAccCols;
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 16) {
+        if (c0 >= item.valid) break;
+        uint32_t g[16], u[16];
+        tmem_ld_x16(t0 + c0, g);
+        if (KIND == 0) tmem_ld_x16(t0 + BN + c0, u);
+        tmem_ld_wait();
+        if (KIND == 0) {
+          __nv_bfloat16* dst = a.h + static_cast<size_t>(item.q0 + c0) * a.I + ch;
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c0 + j < item.valid)
+              dst[static_cast<size_t>(j) * a.I] = __float2bfloat16_rn(silu_mul(__uint_as_float(g[j]), __uint_as_float(u[j])));
+        } else {
+          float* dst = a.y + static_cast<size_t>(item.q0 + c0) * a.H + ch;
+          const float* wq = a.w_sorted + item.q0 + c0;
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c0 + j < item.valid) dst[static_cast<size_t>(j) * a.H] = __ldg(wq + j) * __uint_as_float(g[j]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
+    }
+  }
+
+  // ---------------- teardown ----------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem_base, C::kTmemCols);
+  }
+  if (tid == 0 && *s_abort) atomicOr(a.status, DAMOE_STATUS_WAIT_TIMEOUT);
+}
+
+template <int KIND, int V>
+struct VCfg {
+  static constexpr int kBN = variant_desc(V).tile_n;
+  static constexpr int kStages = (KIND == 0) ? variant_desc(V).stages13 : variant_desc(V).stages2;
+  using C = Cfg<KIND, kBN, kStages>;
+};
+
+}  // namespace
+}  // namespace damoe

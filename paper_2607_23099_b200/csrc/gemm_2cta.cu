@@ -16,9 +16,7 @@
 //
 // Every mbarrier wait is bounded; the only unbounded synchronisation is the cluster barrier at
 // start-up and at teardown, which both CTAs always reach.
-#include "common.cuh"
-#include "gemm_common.cuh"
-#include "ptx.cuh"
+#include "gemm_1cta.cuh"
 
 namespace damoe {
 
@@ -293,15 +291,31 @@ template <int KIND>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
     gemm2_branch_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
   extern __shared__ uint8_t smem_raw[];
+  // One launch covers the whole family: the 1-CTA variants simply ignore that they were
+  // launched as clusters of two, the CTA-pair variants use it.
   const int v = *a.variant_id;
-  if (v == 5) gemm2_body<KIND, VCfg2<KIND, 5>::kBN, VCfg2<KIND, 5>::kStages>(&maps.w, &maps.act[2], a, 5, smem_raw);
-  else if (v == 6) gemm2_body<KIND, VCfg2<KIND, 6>::kBN, VCfg2<KIND, 6>::kStages>(&maps.w, &maps.act[3], a, 6, smem_raw);
+  switch (v) {
+    case 0: gemm_body<KIND, VCfg<KIND, 0>::kBN, VCfg<KIND, 0>::kStages>(&maps.w, &maps.act[0], a, 0, smem_raw); break;
+    case 1: gemm_body<KIND, VCfg<KIND, 1>::kBN, VCfg<KIND, 1>::kStages>(&maps.w, &maps.act[1], a, 1, smem_raw); break;
+    case 2: gemm_body<KIND, VCfg<KIND, 2>::kBN, VCfg<KIND, 2>::kStages>(&maps.w, &maps.act[2], a, 2, smem_raw); break;
+    case 3: gemm_body<KIND, VCfg<KIND, 3>::kBN, VCfg<KIND, 3>::kStages>(&maps.w, &maps.act[3], a, 3, smem_raw); break;
+    case 4: gemm_body<KIND, VCfg<KIND, 4>::kBN, VCfg<KIND, 4>::kStages>(&maps.w, &maps.act[4], a, 4, smem_raw); break;
+    case 5: gemm2_body<KIND, VCfg2<KIND, 5>::kBN, VCfg2<KIND, 5>::kStages>(&maps.w, &maps.act[2], a, 5, smem_raw); break;
+    case 6: gemm2_body<KIND, VCfg2<KIND, 6>::kBN, VCfg2<KIND, 6>::kStages>(&maps.w, &maps.act[3], a, 6, smem_raw); break;
+    default: break;
+  }
 }
 
 template <int KIND>
 constexpr int max_smem2() {
-  return VCfg2<KIND, 5>::C::kSmemBytes > VCfg2<KIND, 6>::C::kSmemBytes ? VCfg2<KIND, 5>::C::kSmemBytes
-                                                                       : VCfg2<KIND, 6>::C::kSmemBytes;
+  int m = VCfg2<KIND, 5>::C::kSmemBytes > VCfg2<KIND, 6>::C::kSmemBytes ? VCfg2<KIND, 5>::C::kSmemBytes
+                                                                        : VCfg2<KIND, 6>::C::kSmemBytes;
+  m = VCfg<KIND, 0>::C::kSmemBytes > m ? VCfg<KIND, 0>::C::kSmemBytes : m;
+  m = VCfg<KIND, 1>::C::kSmemBytes > m ? VCfg<KIND, 1>::C::kSmemBytes : m;
+  m = VCfg<KIND, 2>::C::kSmemBytes > m ? VCfg<KIND, 2>::C::kSmemBytes : m;
+  m = VCfg<KIND, 3>::C::kSmemBytes > m ? VCfg<KIND, 3>::C::kSmemBytes : m;
+  m = VCfg<KIND, 4>::C::kSmemBytes > m ? VCfg<KIND, 4>::C::kSmemBytes : m;
+  return m;
 }
 
 template <int KIND, int V>

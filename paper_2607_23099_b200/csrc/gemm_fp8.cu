@@ -247,20 +247,25 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
         }
         tc_fence_after();
         const uint32_t t0 = tmem_base + (lane_base << 16) + pb * C::kAccCols + col0;
-        if (col0 < item.valid) {
-          float p[CW];
-          tmem_ld_cols<CW>(t0, p);
+        // only the 16-column (8 for the narrowest tile) chunks that hold valid tokens are promoted
+        constexpr int CH = CW < 16 ? CW : 16;
 #pragma unroll
-          for (int j = 0; j < CW; ++j) {
-            const float sx = __shfl_sync(0xffffffffu, (j < 32) ? sx0 : sx1, j & 31);
-            acc_g[j] = fmaf(p[j], sx * swg, acc_g[j]);
-          }
-          if (KIND == 0) {
-            tmem_ld_cols<CW>(t0 + BN, p);
+        for (int c = 0; c < CW; c += CH) {
+          if (col0 + c < item.valid) {  // warp-uniform
+            float p[CH];
+            tmem_ld_cols<CH>(t0 + c, p);
 #pragma unroll
-            for (int j = 0; j < CW; ++j) {
-              const float sx = __shfl_sync(0xffffffffu, (j < 32) ? sx0 : sx1, j & 31);
-              acc_u[j] = fmaf(p[j], sx * swu, acc_u[j]);
+            for (int j = 0; j < CH; ++j) {
+              const float sx = __shfl_sync(0xffffffffu, (c + j < 32) ? sx0 : sx1, (c + j) & 31);
+              acc_g[c + j] = fmaf(p[j], sx * swg, acc_g[c + j]);
+            }
+            if (KIND == 0) {
+              tmem_ld_cols<CH>(t0 + BN + c, p);
+#pragma unroll
+              for (int j = 0; j < CH; ++j) {
+                const float sx = __shfl_sync(0xffffffffu, (c + j < 32) ? sx0 : sx1, (c + j) & 31);
+                acc_u[c + j] = fmaf(p[j], sx * swu, acc_u[c + j]);
+              }
             }
           }
         }
@@ -277,9 +282,11 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
         float hb[CW];
 #pragma unroll
         for (int j = 0; j < CW; ++j) {
-          hb[j] = __bfloat162float(__float2bfloat16_rn(silu_mul(acc_g[j], acc_u[j])));
-          const unsigned m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(hb[j])));
-          if (lane == 0) xa[quad * BN + col0 + j] = __uint_as_float(m);
+          if (col0 + j < item.valid) {  // warp-uniform
+            hb[j] = __bfloat162float(__float2bfloat16_rn(silu_mul(acc_g[j], acc_u[j])));
+            const unsigned m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(hb[j])));
+            if (lane == 0) xa[quad * BN + col0 + j] = __uint_as_float(m);
+          }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_xchg + 8u * half);
