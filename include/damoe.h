@@ -142,7 +142,12 @@ int damoe_route_stats_noalloc(const int32_t* topk_ids, int T, int k, int E, int3
  * DAMOE_VARIANT_AUTO, or DAMOE_VARIANT_STATIC.  The token-count bucket is the smallest table
  * bucket >= T, else the largest (T is a host-known shape, so this costs no synchronisation).
  * Enqueues on `stream`; never synchronises; safe to capture in a CUDA graph unless the
- * dispatch mode is DAMOE_DISPATCH_GRAPH_SWITCH (which launches an internal graph).
+ * dispatch mode is DAMOE_DISPATCH_GRAPH_SWITCH.  In that mode a DAMOE_VARIANT_AUTO call runs as
+ * an internal CUDA graph - route + gather kernels, a conditional SWITCH node whose body v holds
+ * the two GEMMs of variant v and which the selector kernel drives with cudaGraphSetConditional,
+ * then the reduce - launched on `stream`; the graph is rebuilt when any pointer, T, or the
+ * table bucket differs from the previous call and reused otherwise, and `stream` must not be
+ * capturing.
  * Calls on one context must not overlap on the GPU: they share the context's workspace.
  */
 int damoe_fused_moe(damoe_ctx* ctx, const void* x, const void* w13, const void* w2,

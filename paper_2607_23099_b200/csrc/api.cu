@@ -43,6 +43,19 @@ struct damoe_ctx {
   int num_variants() const { return dtype != DAMOE_BF16 ? kNumVariantsFp8 : pairs_ok ? kNumVariants : kNumVariants1Cta; }
   // staging for the host-buffer entry point
   void *st_x = nullptr, *st_ids = nullptr, *st_w = nullptr, *st_out = nullptr;
+  // DAMOE_DISPATCH_GRAPH_SWITCH: the last layer call as a graph with a conditional SWITCH node
+  struct SwitchKey {
+    const void *x = nullptr, *w13 = nullptr, *w2 = nullptr, *ids = nullptr, *wts = nullptr, *out = nullptr;
+    const void *xs = nullptr, *w13s = nullptr, *w2s = nullptr, *bucket = nullptr;
+    int T = -1, mode = -1;
+    bool operator==(const SwitchKey& o) const {
+      return x == o.x && w13 == o.w13 && w2 == o.w2 && ids == o.ids && wts == o.wts && out == o.out && xs == o.xs &&
+             w13s == o.w13s && w2s == o.w2s && bucket == o.bucket && T == o.T && mode == o.mode;
+    }
+  } sw_key;
+  cudaGraph_t sw_graph = nullptr;
+  cudaGraphExec_t sw_exec = nullptr;
+  cudaStream_t cap_stream = nullptr;
   // stage timing
   bool profiling = false;
   cudaEvent_t ev[128][6] = {};
@@ -187,6 +200,127 @@ struct Reader {
   }
 };
 
+
+struct LaunchPack {
+  GemmMaps m13, m2;
+  GemmArgs ga;
+  GemmArgs8 g13, g2;
+};
+
+void build_pack(const damoe_ctx* c, LaunchPack* p) {
+  p->m13.w = c->map_w13;
+  p->m2.w = c->map_w2;
+  for (int v = 0; v < kNumVariants; ++v) {
+    p->m13.act[v] = c->map_x[v];
+    p->m2.act[v] = c->map_h[v];
+  }
+  GemmArgs ga{};
+  ga.ntile_prefix = c->ws.ntile_prefix;
+  ga.offsets = c->ws.offsets;
+  ga.variant_id = c->ws.variant_id;
+  ga.status = c->ws.status;
+  ga.w_sorted = c->ws.w_sorted;
+  ga.h = c->ws.h;
+  ga.y = c->ws.y;
+  ga.E = c->E; ga.H = c->H; ga.I = c->I;
+  p->ga = ga;
+  GemmArgs8 g13{}, g2{};
+  g13.ntile_prefix = g2.ntile_prefix = c->ws.ntile_prefix;
+  g13.offsets = g2.offsets = c->ws.offsets;
+  g13.variant_id = g2.variant_id = c->ws.variant_id;
+  g13.status = g2.status = c->ws.status;
+  g13.w_sorted = g2.w_sorted = c->ws.w_sorted;
+  g13.hq = g2.hq = c->ws.hq;
+  g13.hs_T = g2.hs_T = c->ws.hs_T;
+  g13.y = g2.y = c->ws.y;
+  g13.E = g2.E = c->E; g13.H = g2.H = c->H; g13.I = g2.I = c->I; g13.max_P = g2.max_P = c->max_P;
+  g13.w_scale = c->w13_scale; g13.act_scale_T = c->ws.xs_T;
+  g2.w_scale = c->w2_scale; g2.act_scale_T = c->ws.hs_T;
+  p->g13 = g13;
+  p->g2 = g2;
+}
+
+// One GEMM (kind 0 = gate/up, 1 = down) of one fixed variant, or predicated on the device-side id.
+cudaError_t enqueue_gemm(const damoe_ctx* c, const LaunchPack& p, int kind, int v, bool predicated, cudaStream_t st) {
+  const GemmMaps& maps = kind == 0 ? p.m13 : p.m2;
+  if (c->dtype != DAMOE_BF16) return launch_gemm8(kind, v, predicated, maps, kind == 0 ? p.g13 : p.g2, c->sm_count, st);
+  if (v >= kNumVariants1Cta) return launch_gemm2cta(kind, v, predicated, maps, p.ga, c->sm_count, st);
+  return launch_gemm(kind, v, predicated, maps, p.ga, c->sm_count, st);
+}
+
+cudaError_t enqueue_gather(const damoe_ctx* c, const void* x, int T, cudaStream_t st) {
+  if (c->dtype != DAMOE_BF16)
+    return launch_gather8(c->ws, static_cast<const uint8_t*>(x), c->x_scale, T, c->k, c->H, st);
+  return launch_gather(c->ws, static_cast<const __nv_bfloat16*>(x), T, c->k, c->H, st);
+}
+
+// Builds (or reuses) the layer as one CUDA graph: route + gather, a conditional SWITCH node
+// whose body v holds the two GEMMs of variant v, then the reduce (paper Section IV-C).
+int graph_switch_call(damoe_ctx* c, const void* x, const int32_t* ids, const float* wts, int T, void* out,
+                      SelectorArgs sel, const LaunchPack& pack, cudaStream_t st) {
+  damoe_ctx::SwitchKey key;
+  key.x = x; key.w13 = c->cached_w13; key.w2 = c->cached_w2; key.ids = ids; key.wts = wts; key.out = out;
+  key.xs = c->x_scale; key.w13s = c->w13_scale; key.w2s = c->w2_scale;
+  key.bucket = sel.mode == DAMOE_MODE_EXEMPLAR ? static_cast<const void*>(sel.exemplars)
+               : sel.mode == DAMOE_MODE_EFFEXP_BINS ? static_cast<const void*>(sel.bin_variant)
+                                                    : static_cast<const void*>(sel.cost);
+  key.T = T; key.mode = sel.mode;
+  if (!c->sw_exec || !(key == c->sw_key)) {
+    if (c->sw_exec) cudaGraphExecDestroy(c->sw_exec);
+    if (c->sw_graph) cudaGraphDestroy(c->sw_graph);
+    c->sw_exec = nullptr;
+    c->sw_graph = nullptr;
+    if (!c->cap_stream) DAMOE_CUDA(c, cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking));
+    cudaStream_t cs = c->cap_stream;
+    cudaGraph_t g = nullptr, tmp = nullptr;
+    DAMOE_CUDA(c, cudaGraphCreate(&g, 0));
+    c->sw_graph = g;
+    cudaGraphConditionalHandle handle;
+    DAMOE_CUDA(c, cudaGraphConditionalHandleCreate(&handle, g, 0, cudaGraphCondAssignDefault));
+    sel.cond_handle = handle;
+    sel.use_cond = 1;
+    const cudaStreamCaptureMode mode = cudaStreamCaptureModeThreadLocal;
+    // head: routing metadata + selection (sets the handle) + token gather
+    DAMOE_CUDA(c, cudaStreamBeginCaptureToGraph(cs, g, nullptr, nullptr, 0, mode));
+    cudaError_t e1 = launch_route(c->ws, ids, wts, T, c->k, c->E, sel, nullptr, nullptr, false, cs);
+    cudaError_t e2 = enqueue_gather(c, x, T, cs);
+    cudaStreamCaptureStatus cst;
+    const cudaGraphNode_t* deps = nullptr;
+    size_t ndeps = 0;
+    cudaError_t e3 = cudaStreamGetCaptureInfo(cs, &cst, nullptr, nullptr, &deps, &ndeps);
+    std::vector<cudaGraphNode_t> head(deps, deps + (e3 == cudaSuccess ? ndeps : 0));
+    cudaError_t e4 = cudaStreamEndCapture(cs, &tmp);
+    if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess)
+      return fail(c, DAMOE_ERR_CUDA, "capturing the head of the dispatch graph failed");
+    // the SWITCH node: body v = both GEMMs of variant v
+    const int nv = c->num_variants();
+    cudaGraphNodeParams cp{};
+    cp.type = cudaGraphNodeTypeConditional;
+    cp.conditional.handle = handle;
+    cp.conditional.type = cudaGraphCondTypeSwitch;
+    cp.conditional.size = static_cast<unsigned int>(nv);
+    cudaGraphNode_t cond;
+    DAMOE_CUDA(c, cudaGraphAddNode(&cond, g, head.data(), head.size(), &cp));
+    for (int v = 0; v < nv; ++v) {
+      DAMOE_CUDA(c, cudaStreamBeginCaptureToGraph(cs, cp.conditional.phGraph_out[v], nullptr, nullptr, 0, mode));
+      cudaError_t a = enqueue_gemm(c, pack, 0, v, false, cs);
+      cudaError_t b = enqueue_gemm(c, pack, 1, v, false, cs);
+      cudaError_t d = cudaStreamEndCapture(cs, &tmp);
+      if (a != cudaSuccess || b != cudaSuccess || d != cudaSuccess)
+        return fail(c, DAMOE_ERR_CUDA, "capturing body %d of the dispatch graph failed", v);
+    }
+    // tail: unpermute-reduce after whichever body ran
+    DAMOE_CUDA(c, cudaStreamBeginCaptureToGraph(cs, g, &cond, nullptr, 1, mode));
+    cudaError_t t1 = launch_reduce(c->ws, static_cast<__nv_bfloat16*>(out), T, c->k, c->H, cs);
+    cudaError_t t2 = cudaStreamEndCapture(cs, &tmp);
+    if (t1 != cudaSuccess || t2 != cudaSuccess) return fail(c, DAMOE_ERR_CUDA, "capturing the tail of the dispatch graph failed");
+    DAMOE_CUDA(c, cudaGraphInstantiate(&c->sw_exec, g, 0));
+    c->sw_key = key;
+  }
+  DAMOE_CUDA(c, cudaGraphLaunch(c->sw_exec, st));
+  return DAMOE_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -302,6 +436,9 @@ int damoe_destroy(damoe_ctx* c) {
   for (auto& set : c->ev)
     for (auto& e : set)
       if (e) cudaEventDestroy(e);
+  if (c->sw_exec) cudaGraphExecDestroy(c->sw_exec);
+  if (c->sw_graph) cudaGraphDestroy(c->sw_graph);
+  if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
   if (c->arena) cudaFree(c->arena);
   if (c->table_blob) cudaFree(c->table_blob);
   delete c;
@@ -310,7 +447,7 @@ int damoe_destroy(damoe_ctx* c) {
 
 int damoe_set_dispatch(damoe_ctx* c, int mode) {
   if (!c) return DAMOE_ERR_INVALID_ARG;
-  if (mode != DAMOE_DISPATCH_BRANCH && mode != DAMOE_DISPATCH_PREDICATED)
+  if (mode != DAMOE_DISPATCH_BRANCH && mode != DAMOE_DISPATCH_PREDICATED && mode != DAMOE_DISPATCH_GRAPH_SWITCH)
     return fail(c, DAMOE_ERR_INVALID_ARG, "dispatch mode %d is not available", mode);
   c->dispatch = mode;
   return DAMOE_OK;
@@ -461,86 +598,37 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
   if (ev) DAMOE_CUDA(c, cudaEventRecord(ev[i], st))
   SelectorArgs sel;
   const int known = make_selector(c, T, variant, &sel);
+  LaunchPack pack;
+  build_pack(c, &pack);
+  if (known < 0 && c->dispatch == DAMOE_DISPATCH_GRAPH_SWITCH)
+    return graph_switch_call(c, x, topk_ids, topk_weights, T, out, sel, pack, st);
   DAMOE_MARK(0);
   DAMOE_CUDA(c, launch_route(c->ws, topk_ids, topk_weights, T, c->k, c->E, sel, nullptr, nullptr, false, st));
   DAMOE_MARK(1);
-  if (fp8)
-    DAMOE_CUDA(c, launch_gather8(c->ws, static_cast<const uint8_t*>(x), c->x_scale, T, c->k, c->H, st));
-  else
-    DAMOE_CUDA(c, launch_gather(c->ws, static_cast<const __nv_bfloat16*>(x), T, c->k, c->H, st));
+  DAMOE_CUDA(c, enqueue_gather(c, x, T, st));
   DAMOE_MARK(2);
 
-  GemmMaps m13, m2;
-  m13.w = c->map_w13;
-  m2.w = c->map_w2;
-  for (int v = 0; v < kNumVariants; ++v) {
-    m13.act[v] = c->map_x[v];
-    m2.act[v] = c->map_h[v];
-  }
-  GemmArgs ga{};
-  ga.ntile_prefix = c->ws.ntile_prefix;
-  ga.offsets = c->ws.offsets;
-  ga.variant_id = c->ws.variant_id;
-  ga.status = c->ws.status;
-  ga.w_sorted = c->ws.w_sorted;
-  ga.h = c->ws.h;
-  ga.y = c->ws.y;
-  ga.E = c->E; ga.H = c->H; ga.I = c->I;
-
-  GemmArgs8 g13{}, g2{};
-  g13.ntile_prefix = g2.ntile_prefix = c->ws.ntile_prefix;
-  g13.offsets = g2.offsets = c->ws.offsets;
-  g13.variant_id = g2.variant_id = c->ws.variant_id;
-  g13.status = g2.status = c->ws.status;
-  g13.w_sorted = g2.w_sorted = c->ws.w_sorted;
-  g13.hq = g2.hq = c->ws.hq;
-  g13.hs_T = g2.hs_T = c->ws.hs_T;
-  g13.y = g2.y = c->ws.y;
-  g13.E = g2.E = c->E; g13.H = g2.H = c->H; g13.I = g2.I = c->I; g13.max_P = g2.max_P = c->max_P;
-  g13.w_scale = c->w13_scale; g13.act_scale_T = c->ws.xs_T;
-  g2.w_scale = c->w2_scale; g2.act_scale_T = c->ws.hs_T;
-
-  if (fp8) {
-    if (known >= 0) {
-      DAMOE_CUDA(c, launch_gemm8(0, known, false, m13, g13, c->sm_count, st));
-      DAMOE_MARK(3);
-      DAMOE_CUDA(c, launch_gemm8(1, known, false, m2, g2, c->sm_count, st));
-    } else if (c->dispatch == DAMOE_DISPATCH_PREDICATED) {
-      for (int v = 0; v < kNumVariantsFp8; ++v) DAMOE_CUDA(c, launch_gemm8(0, v, true, m13, g13, c->sm_count, st));
-      DAMOE_MARK(3);
-      for (int v = 0; v < kNumVariantsFp8; ++v) DAMOE_CUDA(c, launch_gemm8(1, v, true, m2, g2, c->sm_count, st));
-    } else {
-      DAMOE_CUDA(c, launch_gemm8(0, -1, false, m13, g13, c->sm_count, st));
-      DAMOE_MARK(3);
-      DAMOE_CUDA(c, launch_gemm8(1, -1, false, m2, g2, c->sm_count, st));
-    }
-  } else if (known >= 0) {
-    if (known >= kNumVariants1Cta) {
-      DAMOE_CUDA(c, launch_gemm2cta(0, known, false, m13, ga, c->sm_count, st));
-      DAMOE_MARK(3);
-      DAMOE_CUDA(c, launch_gemm2cta(1, known, false, m2, ga, c->sm_count, st));
-    } else {
-      DAMOE_CUDA(c, launch_gemm(0, known, false, m13, ga, c->sm_count, st));
-      DAMOE_MARK(3);
-      DAMOE_CUDA(c, launch_gemm(1, known, false, m2, ga, c->sm_count, st));
-    }
+  if (known >= 0) {
+    DAMOE_CUDA(c, enqueue_gemm(c, pack, 0, known, false, st));
+    DAMOE_MARK(3);
+    DAMOE_CUDA(c, enqueue_gemm(c, pack, 1, known, false, st));
   } else if (c->dispatch == DAMOE_DISPATCH_PREDICATED) {
     const int nv = c->num_variants();
-    for (int v = 0; v < nv; ++v)
-      DAMOE_CUDA(c, v < kNumVariants1Cta ? launch_gemm(0, v, true, m13, ga, c->sm_count, st)
-                                         : launch_gemm2cta(0, v, true, m13, ga, c->sm_count, st));
+    for (int v = 0; v < nv; ++v) DAMOE_CUDA(c, enqueue_gemm(c, pack, 0, v, true, st));
     DAMOE_MARK(3);
-    for (int v = 0; v < nv; ++v)
-      DAMOE_CUDA(c, v < kNumVariants1Cta ? launch_gemm(1, v, true, m2, ga, c->sm_count, st)
-                                         : launch_gemm2cta(1, v, true, m2, ga, c->sm_count, st));
+    for (int v = 0; v < nv; ++v) DAMOE_CUDA(c, enqueue_gemm(c, pack, 1, v, true, st));
+  } else if (fp8) {
+    DAMOE_CUDA(c, launch_gemm8(0, -1, false, pack.m13, pack.g13, c->sm_count, st));
+    DAMOE_MARK(3);
+    DAMOE_CUDA(c, launch_gemm8(1, -1, false, pack.m2, pack.g2, c->sm_count, st));
   } else {
     // one persistent kernel per GEMM that branches on the variant id; when the CTA-pair variants
     // exist it is launched as clusters of two so that it can hold the whole family
-    if (c->pairs_ok) DAMOE_CUDA(c, launch_gemm2cta(0, -2, false, m13, ga, c->sm_count, st));
-    else DAMOE_CUDA(c, launch_gemm(0, -1, false, m13, ga, c->sm_count, st));
+    if (c->pairs_ok) DAMOE_CUDA(c, launch_gemm2cta(0, -2, false, pack.m13, pack.ga, c->sm_count, st));
+    else DAMOE_CUDA(c, launch_gemm(0, -1, false, pack.m13, pack.ga, c->sm_count, st));
     DAMOE_MARK(3);
-    if (c->pairs_ok) DAMOE_CUDA(c, launch_gemm2cta(1, -2, false, m2, ga, c->sm_count, st));
-    else DAMOE_CUDA(c, launch_gemm(1, -1, false, m2, ga, c->sm_count, st));
+    if (c->pairs_ok) DAMOE_CUDA(c, launch_gemm2cta(1, -2, false, pack.m2, pack.ga, c->sm_count, st));
+    else DAMOE_CUDA(c, launch_gemm(1, -1, false, pack.m2, pack.ga, c->sm_count, st));
   }
   DAMOE_MARK(4);
   DAMOE_CUDA(c, launch_reduce(c->ws, static_cast<__nv_bfloat16*>(out), T, c->k, c->H, st));

@@ -45,6 +45,8 @@ struct SelectorArgs {
   uint64_t bin_den;
   const int32_t* bin_variant;  // [n_bins]
   const int64_t* cost;         // COST: [4, V] = c_fix, c_byte, c_reload, c_flop
+  unsigned long long cond_handle;  // CUDA-graph conditional handle the chosen id is also written to ...
+  int use_cond;                    // ... when non-zero (DAMOE_DISPATCH_GRAPH_SWITCH)
 };
 
 // Pointers into the context's workspace that the kernels use.

@@ -163,7 +163,10 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
 
   // ---- selector ------------------------------------------------------------------
   if (sel.forced >= 0) {
-    if (tid == 0) *ws.variant_id = sel.forced;
+    if (tid == 0) {
+      *ws.variant_id = sel.forced;
+      if (sel.use_cond) cudaGraphSetConditional(sel.cond_handle, static_cast<unsigned int>(sel.forced));
+    }
     return;
   }
   int chosen = 0;
@@ -224,6 +227,8 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
       chosen = 0;
     }
     *ws.variant_id = chosen;
+    // the same id drives the SWITCH node when the layer runs as a conditional CUDA graph
+    if (sel.use_cond) cudaGraphSetConditional(sel.cond_handle, static_cast<unsigned int>(chosen));
   }
 }
 

@@ -198,6 +198,43 @@ def test_selected_variant_matches_oracle_given_the_same_table(d):
     m.close()
 
 
+def test_graph_switch_dispatch(d):
+    # the conditional-graph SWITCH path: same results and same choices as the in-kernel branch,
+    # with the graph reused while the buffers stay the same and the routing inside them changes
+    from paper_2607_23099_b200 import tuning
+    E, k, H, I, T = 8, 2, 1024, 512, 96
+    V, ns = d.variant_count(), d.tile_ns()
+    W = di.MoEWeights(3, E, H, I)
+    w13, w2 = W.materialize("cuda")
+    table = _table_for(E, k, [128], d.MODE_EXEMPLAR, V, ns)
+    m = d.DAMoE(128, k, E, H, I)
+    m.load_tuning_table(tuning.pack_table(table, E, k, H, I, d.BF16, V))
+    ids_d = torch.empty(T, k, dtype=torch.int32, device="cuda")
+    w_d = torch.empty(T, k, dtype=torch.float32, device="cuda")
+    x_d = torch.empty(T, H, dtype=torch.bfloat16, device="cuda")
+    out = torch.empty(T, H, dtype=torch.bfloat16, device="cuda")
+    chosen = set()
+    for seed, alpha in [(1, 0.05), (2, 10.0), (3, 0.2), (4, 1.0)]:
+        case = Case(seed, T, E, k, H, I, alpha)
+        case.weights = W
+        ids_d.copy_(torch.from_numpy(case.ids))
+        w_d.copy_(torch.from_numpy(case.w))
+        x_d.copy_(case.x("cuda"))
+        m.set_dispatch(d.DISPATCH_BRANCH)
+        ref_out = m.fused_moe(x_d, w13, w2, ids_d, w_d, d.VARIANT_AUTO).clone()
+        ref_meta = m.debug_fetch(T)
+        m.set_dispatch(d.DISPATCH_GRAPH_SWITCH)
+        m.fused_moe(x_d, w13, w2, ids_d, w_d, d.VARIANT_AUTO, out=out)
+        meta = m.debug_fetch(T)
+        assert meta["status"] == 0
+        assert meta["variant_id"] == ref_meta["variant_id"] == route.select_variant(table, route.histogram(case.ids, E), T, ns)
+        assert torch.equal(out.view(torch.int16), ref_out.view(torch.int16))
+        _check_layer(out, case)
+        chosen.add(meta["variant_id"])
+    assert len(chosen) >= 2
+    m.close()
+
+
 def test_host_buffer_entry_point(d):
     case = config0(seed=6, T=32)
     t = _device_case(case)
