@@ -289,6 +289,48 @@ def compare_dispatch(m, d, cells, run, pk, reps=3):
                 layer_roofline_frac_min=round(min(r["roofline_frac"] for r in rows), 4), batches=len(rows)), rows
 
 
+def dispatch_overhead(m, d, w13, w2, device, reps=30):
+    """Microseconds per layer at T = 1 and T = 8 for: a fixed variant (no selection), the static
+    bucket choice, and AUTO through each dispatch mechanism (in-kernel branch, predicated
+    launches, conditional-graph SWITCH); plus the paper's Table III microbenchmark re-measured."""
+    w = WORKLOAD
+    stream = torch.cuda.current_stream()
+    out = {}
+    for T in (1, 8):
+        ids, wts, _ = di.routing_batch(4242 + T, T, w["k"], w["E"], 1.0)
+        x = di.activations(4242 + T, T, w["H"], device)
+        ids_d, w_d = torch.from_numpy(ids).to(device), torch.from_numpy(wts).to(device)
+        o = torch.empty(T, w["H"], dtype=torch.bfloat16, device=device)
+
+        def timed(variant):
+            for _ in range(3):
+                m.fused_moe(x, w13, w2, ids_d, w_d, variant, out=o, stream=stream)
+            ts = []
+            for _ in range(reps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                m.fused_moe(x, w13, w2, ids_d, w_d, variant, out=o, stream=stream)
+                b.record(stream)
+                b.synchronize()
+                ts.append(a.elapsed_time(b) * 1e3)
+            return round(statistics.median(ts), 1)
+
+        row = {}
+        m.set_dispatch(d.DISPATCH_BRANCH)
+        row["auto_branch_us"] = timed(d.VARIANT_AUTO)
+        chosen = m.debug_fetch(T)["variant_id"]
+        row["fixed_variant_us"] = timed(chosen)
+        row["static_us"] = timed(d.VARIANT_STATIC)
+        m.set_dispatch(d.DISPATCH_PREDICATED)
+        row["auto_predicated_us"] = timed(d.VARIANT_AUTO)
+        m.set_dispatch(d.DISPATCH_GRAPH_SWITCH)
+        row["auto_graph_switch_us"] = timed(d.VARIANT_AUTO)
+        m.set_dispatch(d.DISPATCH_BRANCH)
+        out[f"T{T}"] = row
+    out["microbench_us"] = {k: round(v, 2) for k, v in d.dispatch_microbench(200, device.index or 0).items()}
+    return out
+
+
 def run_ours(args):
     import paper_2607_23099_b200 as d
 
@@ -390,6 +432,11 @@ def run_ours(args):
         tsum, trows = compare_dispatch(m, d, tcells, run, pk)
         dispatch["trace"] = dict(tsum, what="48 batches, T log-uniform [1, 64], alpha log-uniform [0.05, 10]")
 
+    # ---- cost of keeping the decision on the device: the three dispatch mechanisms at small T ----
+    overhead = None
+    if args.workload == "headline" and not fp8:
+        overhead = dispatch_overhead(m, d, w13, w2, device)
+
     if rank != 0:
         return
 
@@ -437,7 +484,7 @@ def run_ours(args):
                 aggregate_layers_per_s=round(world * 1e6 / us_per_layer, 2),
                 e2e=dict(value=round(e2e_us, 2), unit="us", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
                 gpu_launches=7 * steps, clocks=clocks, roofline=roofline, cpu_baseline=cpu, dispatch=dispatch,
-                device_status=status)
+                dispatch_overhead=overhead, device_status=status)
     print(json.dumps(line))
 
 

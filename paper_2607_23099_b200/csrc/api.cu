@@ -2,6 +2,7 @@
 // call.  The host side only validates, picks the token-count bucket from T (a shape the host
 // knows) and enqueues kernels; every routing-dependent decision is taken on the device.
 #include <cstdarg>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -280,6 +281,11 @@ int graph_switch_call(damoe_ctx* c, const void* x, const int32_t* ids, const flo
     sel.cond_handle = handle;
     sel.use_cond = 1;
     const cudaStreamCaptureMode mode = cudaStreamCaptureModeThreadLocal;
+    struct PdlOff {  // plain serial edges inside the dispatch graph: programmatic edges do not cross a conditional node
+      bool saved = g_pdl;
+      PdlOff() { g_pdl = false; }
+      ~PdlOff() { g_pdl = saved; }
+    } pdl_off;
     // head: routing metadata + selection (sets the handle) + token gather
     DAMOE_CUDA(c, cudaStreamBeginCaptureToGraph(cs, g, nullptr, nullptr, 0, mode));
     cudaError_t e1 = launch_route(c->ws, ids, wts, T, c->k, c->E, sel, nullptr, nullptr, false, cs);
@@ -355,6 +361,7 @@ int damoe_create(damoe_ctx** out, int device, int max_T, int k, int E, int H, in
     damoe_destroy(c);
     return code;
   };
+  if (const char* env = getenv("DAMOE_PDL")) g_pdl = env[0] != '0';
   if (cudaSetDevice(device) != cudaSuccess) return bail(DAMOE_ERR_CUDA);
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return bail(DAMOE_ERR_CUDA);

@@ -8,7 +8,37 @@
 
 #include "../../include/damoe.h"
 
+#include <utility>
+
 namespace damoe {
+
+// Programmatic dependent launch: every kernel of the layer is launched with the
+// programmatic-stream-serialization attribute, lets its successor start early
+// (griddepcontrol.launch_dependents at its top) and waits for its predecessor to have
+// completed (griddepcontrol.wait) before it touches anything the predecessor wrote.  The
+// successor's launch latency and prologue then overlap the predecessor's tail.  Because every
+// kernel waits for the full completion of the one before it, ordering along the chain is kept.
+inline bool g_pdl = true;
+
+template <class... KArgs, class... Args>
+cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = g_pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
 
 constexpr int kMaxE = 1024;
 constexpr int kMaxK = 32;

@@ -34,7 +34,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     gemm_fixed_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_act,
                       const GemmArgs a, const int predicated) {
   extern __shared__ uint8_t smem_raw[];
-  if (predicated && *a.variant_id != V) return;
+  if (predicated) {
+    pdl_launch_dependents();
+    pdl_wait();
+    if (*a.variant_id != V) return;
+  }
   gemm_body<KIND, VCfg<KIND, V>::kBN, VCfg<KIND, V>::kStages>(&tmap_w, &tmap_act, a, V, smem_raw);
 }
 
@@ -42,6 +46,8 @@ template <int KIND>
 __global__ void __launch_bounds__(kGemmThreads, 1)
     gemm_branch_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
   extern __shared__ uint8_t smem_raw[];
+  pdl_launch_dependents();
+  pdl_wait();
   const int v = *a.variant_id;
   switch (v) {
     case 0: gemm_body<KIND, VCfg<KIND, 0>::kBN, VCfg<KIND, 0>::kStages>(&maps.w, &maps.act[0], a, 0, smem_raw); break;
@@ -71,9 +77,8 @@ cudaError_t configure_fixed() {
 
 template <int KIND, int V>
 cudaError_t launch_fixed(const GemmMaps& maps, const GemmArgs& args, bool predicated, int grid, cudaStream_t stream) {
-  gemm_fixed_kernel<KIND, V><<<grid, kGemmThreads, VCfg<KIND, V>::C::kSmemBytes, stream>>>(maps.w, maps.act[V], args,
-                                                                                            predicated ? 1 : 0);
-  return cudaGetLastError();
+  return launch_k(gemm_fixed_kernel<KIND, V>, dim3(grid), dim3(kGemmThreads), VCfg<KIND, V>::C::kSmemBytes, stream,
+                  maps.w, maps.act[V], args, predicated ? 1 : 0);
 }
 
 template <int KIND>
@@ -81,8 +86,7 @@ cudaError_t launch_kind(int variant, bool predicated, const GemmMaps& maps, cons
                         cudaStream_t stream) {
   switch (variant) {
     case -1:
-      gemm_branch_kernel<KIND><<<grid, kGemmThreads, max_smem_bytes<KIND>(), stream>>>(maps, args);
-      return cudaGetLastError();
+      return launch_k(gemm_branch_kernel<KIND>, dim3(grid), dim3(kGemmThreads), max_smem_bytes<KIND>(), stream, maps, args);
     case 0: return launch_fixed<KIND, 0>(maps, args, predicated, grid, stream);
     case 1: return launch_fixed<KIND, 1>(maps, args, predicated, grid, stream);
     case 2: return launch_fixed<KIND, 2>(maps, args, predicated, grid, stream);

@@ -53,6 +53,8 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
+  pdl_launch_dependents();
+  pdl_wait();  // everything below reads what the route / gather / previous GEMM kernels wrote
   const int32_t* pref_g = a.ntile_prefix + variant * (E + 1);
   for (int i = tid; i <= E; i += kGemmThreads) {
     s_pref[i] = pref_g[i];

@@ -121,6 +121,8 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
+  pdl_launch_dependents();
+  pdl_wait();
   const int32_t* pref_g = a.ntile_prefix + variant * (E + 1);
   for (int i = tid; i <= E; i += kThreads2) {
     s_pref[i] = pref_g[i];
@@ -283,7 +285,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
     gemm2_fixed_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_act,
                        const GemmArgs a, const int predicated) {
   extern __shared__ uint8_t smem_raw[];
-  if (predicated && *a.variant_id != V) return;
+  if (predicated) {
+    pdl_launch_dependents();
+    pdl_wait();
+    if (*a.variant_id != V) return;
+  }
   gemm2_body<KIND, VCfg2<KIND, V>::kBN, VCfg2<KIND, V>::kStages>(&tmap_w, &tmap_act, a, V, smem_raw);
 }
 
@@ -293,6 +299,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
   extern __shared__ uint8_t smem_raw[];
   // One launch covers the whole family: the 1-CTA variants simply ignore that they were
   // launched as clusters of two, the CTA-pair variants use it.
+  pdl_launch_dependents();
+  pdl_wait();
   const int v = *a.variant_id;
   switch (v) {
     case 0: gemm_body<KIND, VCfg<KIND, 0>::kBN, VCfg<KIND, 0>::kStages>(&maps.w, &maps.act[0], a, 0, smem_raw); break;
@@ -321,9 +329,8 @@ constexpr int max_smem2() {
 template <int KIND, int V>
 cudaError_t launch_fixed2(const GemmMaps& maps, const GemmArgs& args, bool predicated, int grid, cudaStream_t st) {
   constexpr int kHalfRowsVariant = (VCfg2<KIND, V>::kBN == 128) ? 2 : 3;  // tensor map whose box has N_v / 2 rows
-  gemm2_fixed_kernel<KIND, V><<<grid & ~1, kThreads2, VCfg2<KIND, V>::C::kSmemBytes, st>>>(
-      maps.w, maps.act[kHalfRowsVariant], args, predicated ? 1 : 0);
-  return cudaGetLastError();
+  return launch_k(gemm2_fixed_kernel<KIND, V>, dim3(grid & ~1), dim3(kThreads2), VCfg2<KIND, V>::C::kSmemBytes, st,
+                  maps.w, maps.act[kHalfRowsVariant], args, predicated ? 1 : 0);
 }
 
 }  // namespace
@@ -345,9 +352,9 @@ cudaError_t gemm2cta_configure() {
 cudaError_t launch_gemm2cta(int kind, int variant, bool predicated, const GemmMaps& maps, const GemmArgs& args,
                             int sm_count, cudaStream_t stream) {
   if (variant == -2) {
-    if (kind == 0) gemm2_branch_kernel<0><<<sm_count & ~1, kThreads2, max_smem2<0>(), stream>>>(maps, args);
-    else gemm2_branch_kernel<1><<<sm_count & ~1, kThreads2, max_smem2<1>(), stream>>>(maps, args);
-    return cudaGetLastError();
+    if (kind == 0)
+      return launch_k(gemm2_branch_kernel<0>, dim3(sm_count & ~1), dim3(kThreads2), max_smem2<0>(), stream, maps, args);
+    return launch_k(gemm2_branch_kernel<1>, dim3(sm_count & ~1), dim3(kThreads2), max_smem2<1>(), stream, maps, args);
   }
   if (kind == 0) {
     if (variant == 5) return launch_fixed2<0, 5>(maps, args, predicated, sm_count, stream);

@@ -113,6 +113,8 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
+  pdl_launch_dependents();
+  pdl_wait();
   const int32_t* pref_g = a.ntile_prefix + variant * (E + 1);
   for (int i = tid; i <= E; i += kThreads8) {
     s_pref[i] = pref_g[i];
@@ -341,7 +343,11 @@ __global__ void __launch_bounds__(kThreads8, 1)
     gemm8_fixed_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_act,
                        const GemmArgs8 a, const int predicated) {
   extern __shared__ uint8_t smem_raw[];
-  if (predicated && *a.variant_id != V) return;
+  if (predicated) {
+    pdl_launch_dependents();
+    pdl_wait();
+    if (*a.variant_id != V) return;
+  }
   gemm8_body<KIND, VCfg8<KIND, V>::kBN, VCfg8<KIND, V>::kStages>(&tmap_w, &tmap_act, a, V, smem_raw);
 }
 
@@ -349,6 +355,8 @@ template <int KIND>
 __global__ void __launch_bounds__(kThreads8, 1)
     gemm8_branch_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs8 a) {
   extern __shared__ uint8_t smem_raw[];
+  pdl_launch_dependents();
+  pdl_wait();
   const int v = *a.variant_id;
   switch (v) {
     case 0: gemm8_body<KIND, VCfg8<KIND, 0>::kBN, VCfg8<KIND, 0>::kStages>(&maps.w, &maps.act[0], a, 0, smem_raw); break;
@@ -370,9 +378,8 @@ constexpr int max_smem8() {
 
 template <int KIND, int V>
 cudaError_t launch_fixed8(const GemmMaps& maps, const GemmArgs8& args, bool predicated, int grid, cudaStream_t st) {
-  gemm8_fixed_kernel<KIND, V><<<grid, kThreads8, VCfg8<KIND, V>::C::kSmemBytes, st>>>(maps.w, maps.act[V], args,
-                                                                                      predicated ? 1 : 0);
-  return cudaGetLastError();
+  return launch_k(gemm8_fixed_kernel<KIND, V>, dim3(grid), dim3(kThreads8), VCfg8<KIND, V>::C::kSmemBytes, st, maps.w,
+                  maps.act[V], args, predicated ? 1 : 0);
 }
 
 template <int KIND>
@@ -380,8 +387,7 @@ cudaError_t launch_kind8(int variant, bool predicated, const GemmMaps& maps, con
                          cudaStream_t st) {
   switch (variant) {
     case -1:
-      gemm8_branch_kernel<KIND><<<grid, kThreads8, max_smem8<KIND>(), st>>>(maps, args);
-      return cudaGetLastError();
+      return launch_k(gemm8_branch_kernel<KIND>, dim3(grid), dim3(kThreads8), max_smem8<KIND>(), st, maps, args);
     case 0: return launch_fixed8<KIND, 0>(maps, args, predicated, grid, st);
     case 1: return launch_fixed8<KIND, 1>(maps, args, predicated, grid, st);
     case 2: return launch_fixed8<KIND, 2>(maps, args, predicated, grid, st);
@@ -396,6 +402,8 @@ __global__ void __launch_bounds__(256) gather_rows8_kernel(const uint4* __restri
                                                            const int32_t* __restrict__ perm, int k, int row_vec,
                                                            int nblk, int max_P) {
   const int q = blockIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   const int p = perm[q];
   if (p < 0) return;
   const int t = p / k;
@@ -430,10 +438,9 @@ cudaError_t launch_gemm8(int kind, int variant, bool predicated, const GemmMaps&
 
 cudaError_t launch_gather8(const Workspace& ws, const uint8_t* xq, const float* x_scale, int T, int k, int H,
                            cudaStream_t stream) {
-  gather_rows8_kernel<<<T * k, 256, 0, stream>>>(reinterpret_cast<const uint4*>(xq), x_scale,
-                                                 reinterpret_cast<uint4*>(ws.xq_perm), ws.xs_T, ws.perm, k, H / 16,
-                                                 H / 128, ws.max_P);
-  return cudaGetLastError();
+  return launch_k(gather_rows8_kernel, dim3(T * k), dim3(256), 0, stream, reinterpret_cast<const uint4*>(xq), x_scale,
+                  reinterpret_cast<uint4*>(ws.xq_perm), ws.xs_T, static_cast<const int32_t*>(ws.perm), k, H / 16, H / 128,
+                  ws.max_P);
 }
 
 }  // namespace damoe

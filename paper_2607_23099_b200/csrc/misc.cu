@@ -11,6 +11,8 @@ namespace {
 __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restrict__ x, uint4* __restrict__ x_perm,
                                                           const int32_t* __restrict__ perm, int k, int row_vec) {
   const int q = blockIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   const int p = perm[q];
   if (p < 0) return;
   const uint4* src = x + static_cast<size_t>(p / k) * row_vec;
@@ -25,9 +27,11 @@ __global__ void __launch_bounds__(256) unpermute_reduce_kernel(const float4* __r
                                                                uint2* __restrict__ out, int k, int row_vec) {
   const int t = blockIdx.x;
   __shared__ int s_q[kMaxK];
+  pdl_launch_dependents();
+  pdl_wait();
   if (threadIdx.x < k) s_q[threadIdx.x] = inv[t * k + threadIdx.x];
   __syncthreads();
-  for (int i = threadIdx.x; i < row_vec; i += blockDim.x) {
+  for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < row_vec; i += gridDim.y * blockDim.x) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int j = 0; j < k; ++j) {
       const int q = s_q[j];
@@ -50,15 +54,16 @@ __global__ void __launch_bounds__(256) unpermute_reduce_kernel(const float4* __r
 }  // namespace
 
 cudaError_t launch_gather(const Workspace& ws, const __nv_bfloat16* x, int T, int k, int H, cudaStream_t stream) {
-  gather_rows_kernel<<<T * k, 256, 0, stream>>>(reinterpret_cast<const uint4*>(x), reinterpret_cast<uint4*>(ws.x_perm),
-                                                ws.perm, k, H / 8);
-  return cudaGetLastError();
+  return launch_k(gather_rows_kernel, dim3(T * k), dim3(256), 0, stream, reinterpret_cast<const uint4*>(x),
+                  reinterpret_cast<uint4*>(ws.x_perm), static_cast<const int32_t*>(ws.perm), k, H / 8);
 }
 
 cudaError_t launch_reduce(const Workspace& ws, __nv_bfloat16* out, int T, int k, int H, cudaStream_t stream) {
-  unpermute_reduce_kernel<<<T, 256, 0, stream>>>(reinterpret_cast<const float4*>(ws.y), ws.inv,
-                                                 reinterpret_cast<uint2*>(out), k, H / 4);
-  return cudaGetLastError();
+  // small batches split each row over several CTAs so that more than T SMs pull on the reduction
+  const int row_vec = H / 4;
+  const int split = T >= 512 ? 1 : (row_vec + 255) / 256;
+  return launch_k(unpermute_reduce_kernel, dim3(T, split), dim3(256), 0, stream, reinterpret_cast<const float4*>(ws.y),
+                  static_cast<const int32_t*>(ws.inv), reinterpret_cast<uint2*>(out), k, H / 4);
 }
 
 }  // namespace damoe

@@ -2,7 +2,8 @@
 // (paper Eq. 2), offsets, the stable grouping of (token, slot) pairs by expert, per-variant
 // padded-tile counts, and the device-side choice of the kernel variant (paper Section IV-B).
 //
-// Three small launches:
+// Three small launches (one, the scan kernel in its fused form, when the batch has at most 1024
+// pairs):
 //   count   : one CTA per 512 pairs; warp-aggregated shared-memory histogram -> block_hist[b][e]
 //   scan    : one CTA; scans block_hist over blocks (turning it into per-block bases), writes
 //             hist / sums / eff_exp / offsets / tile prefixes / tile counts, runs the selector
@@ -23,8 +24,10 @@ __global__ void __launch_bounds__(kPairsPerBlock) route_count_kernel(const int32
                                                                      int32_t* __restrict__ block_hist,
                                                                      uint32_t* __restrict__ status) {
   __shared__ int s_hist[kMaxE];
+  pdl_launch_dependents();
   for (int e = threadIdx.x; e < E; e += blockDim.x) s_hist[e] = 0;
   __syncthreads();
+  pdl_wait();
   const int p = blockIdx.x * kPairsPerBlock + threadIdx.x;
   const int lane = threadIdx.x & 31;
   const int e = (p < P) ? ids[p] : -1;
@@ -68,11 +71,20 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int* tot
   return s_warp[warp] + inc - v;
 }
 
+// FUSED = true: the whole routing stage in this one CTA, for batches of at most 1024 pairs (one
+// thread per pair): it counts the histogram itself, and after the offsets are known ranks each
+// pair by brute force over the ids held in shared memory (rank = earlier pairs with the same
+// expert), which gives the same canonical stable order as the three-kernel path.
+template <bool FUSED>
 __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __restrict__ block_hist, int nblocks, int E,
                                                                   Workspace ws, SelectorArgs sel,
                                                                   int32_t* __restrict__ hist_out,
-                                                                  double* __restrict__ eff_out, int stats_only) {
+                                                                  double* __restrict__ eff_out, int stats_only,
+                                                                  const int32_t* __restrict__ ids,
+                                                                  const float* __restrict__ weights, int P) {
   __shared__ int s_hist[kMaxE];
+  __shared__ int s_ids[FUSED ? kScanThreads : 1];
+  __shared__ int s_offs[FUSED ? kMaxE : 1];
   __shared__ int s_sorted[kMaxE];
   __shared__ int s_warp[33];
   __shared__ unsigned long long s_red[2][32];
@@ -80,18 +92,37 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
   __shared__ long long s_score[kMaxExemplars];
   __shared__ int s_active;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_launch_dependents();
+  if (FUSED) {
+    for (int e = tid; e < E; e += kScanThreads) s_hist[e] = 0;
+    __syncthreads();
+  }
+  pdl_wait();
 
-  // per-expert totals; block_hist becomes each block's base inside the expert's segment
-  for (int e = tid; e < E; e += kScanThreads) {
-    int running = 0;
-    for (int b = 0; b < nblocks; ++b) {
-      const int v = block_hist[b * E + e];
-      block_hist[b * E + e] = running;
-      running += v;
+  if (FUSED) {
+    const int e = (tid < P) ? ids[tid] : -1;
+    const bool valid = e >= 0 && e < E;
+    s_ids[tid] = valid ? e : -1;
+    if (tid < P && !valid) atomicOr(ws.status, DAMOE_STATUS_BAD_ID);
+    if (valid) atomicAdd(&s_hist[e], 1);
+    __syncthreads();
+    for (int i = tid; i < E; i += kScanThreads) {
+      if (hist_out) hist_out[i] = s_hist[i];
+      if (!stats_only) ws.hist[i] = s_hist[i];
     }
-    s_hist[e] = running;
-    if (hist_out) hist_out[e] = running;
-    if (!stats_only) ws.hist[e] = running;
+  } else {
+    // per-expert totals; block_hist becomes each block's base inside the expert's segment
+    for (int e = tid; e < E; e += kScanThreads) {
+      int running = 0;
+      for (int b = 0; b < nblocks; ++b) {
+        const int v = block_hist[b * E + e];
+        block_hist[b * E + e] = running;
+        running += v;
+      }
+      s_hist[e] = running;
+      if (hist_out) hist_out[e] = running;
+      if (!stats_only) ws.hist[e] = running;
+    }
   }
   __syncthreads();
 
@@ -139,6 +170,22 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
     const int ex = block_exclusive_scan(t_e, s_warp, &total);
     if (tid < E) ws.offsets[tid] = ex;
     if (tid == 0) ws.offsets[E] = total;
+    if (FUSED) {
+      if (tid < E) s_offs[tid] = ex;
+      __syncthreads();
+      const int e = s_ids[tid];
+      if (e >= 0) {
+        int rank = 0;
+        for (int q = 0; q < tid; ++q) rank += (s_ids[q] == e);
+        const int pos = s_offs[e] + rank;
+        ws.perm[pos] = tid;
+        ws.inv[tid] = pos;
+        ws.w_sorted[pos] = weights[tid];
+      } else if (tid < P) {
+        ws.inv[tid] = -1;
+      }
+      if (tid < P && tid >= total) ws.perm[tid] = -1;  // sorted positions past the valid count
+    }
   }
   // active experts
   {
@@ -238,8 +285,10 @@ __global__ void __launch_bounds__(kPairsPerBlock) route_scatter_kernel(const int
                                                                        Workspace ws) {
   __shared__ unsigned short s_cnt[kWarpsPerRouteBlock][kMaxE];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_launch_dependents();
   for (int i = tid; i < kWarpsPerRouteBlock * E; i += blockDim.x) s_cnt[i / E][i % E] = 0;
   __syncthreads();
+  pdl_wait();
   const int p = blockIdx.x * kPairsPerBlock + tid;
   const int e = (p < P) ? ids[p] : -1;
   const bool valid = (p < P) && e >= 0 && e < E;
@@ -279,12 +328,18 @@ cudaError_t launch_route(const Workspace& ws, const int32_t* topk_ids, const flo
                          cudaStream_t stream) {
   const int P = T * k;
   const int nblocks = (P + kPairsPerBlock - 1) / kPairsPerBlock;
-  route_count_kernel<<<nblocks, kPairsPerBlock, 0, stream>>>(topk_ids, P, E, ws.block_hist, ws.status);
-  route_scan_kernel<<<1, kScanThreads, 0, stream>>>(ws.block_hist, nblocks, E, ws, sel, hist_out, eff_out,
-                                                    stats_only ? 1 : 0);
-  if (!stats_only)
-    route_scatter_kernel<<<nblocks, kPairsPerBlock, 0, stream>>>(topk_ids, topk_weights, P, E, ws.block_hist, ws);
-  return cudaGetLastError();
+  if (P <= kScanThreads && !stats_only)  // small batch: one launch does the whole routing stage
+    return launch_k(route_scan_kernel<true>, dim3(1), dim3(kScanThreads), 0, stream, ws.block_hist, 1, E, ws, sel,
+                    hist_out, eff_out, 0, topk_ids, topk_weights, P);
+  cudaError_t e = launch_k(route_count_kernel, dim3(nblocks), dim3(kPairsPerBlock), 0, stream, topk_ids, P, E,
+                           ws.block_hist, ws.status);
+  if (e != cudaSuccess) return e;
+  e = launch_k(route_scan_kernel<false>, dim3(1), dim3(kScanThreads), 0, stream, ws.block_hist, nblocks, E, ws, sel,
+               hist_out, eff_out, stats_only ? 1 : 0, static_cast<const int32_t*>(nullptr),
+               static_cast<const float*>(nullptr), P);
+  if (e != cudaSuccess || stats_only) return e;
+  return launch_k(route_scatter_kernel, dim3(nblocks), dim3(kPairsPerBlock), 0, stream, topk_ids, topk_weights, P, E,
+                  static_cast<const int32_t*>(ws.block_hist), ws);
 }
 
 }  // namespace damoe
@@ -349,6 +404,6 @@ extern "C" int damoe_route_stats_noalloc(const int32_t* topk_ids, int T, int k, 
   const int P = T * k;
   const int nblocks = (P + kPairsPerBlock - 1) / kPairsPerBlock;
   route_count_kernel<<<nblocks, kPairsPerBlock, 0, st>>>(topk_ids, P, E, ws.block_hist, ws.status);
-  route_scan_kernel<<<1, kScanThreads, 0, st>>>(ws.block_hist, nblocks, E, ws, sel, hist, eff_exp, 1);
+  route_scan_kernel<false><<<1, kScanThreads, 0, st>>>(ws.block_hist, nblocks, E, ws, sel, hist, eff_exp, 1, nullptr, nullptr, P);
   return cudaGetLastError() == cudaSuccess ? DAMOE_OK : DAMOE_ERR_CUDA;
 }

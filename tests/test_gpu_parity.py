@@ -115,6 +115,24 @@ def test_ragged_multi_tile_and_determinism(d):
     m.close()
 
 
+def test_route_metadata_many_pairs(d):
+    # 16 000 pairs: the three-kernel routing path (several 512-pair blocks), integer outputs in full;
+    # 1 024 pairs: the largest batch the single-kernel routing path takes
+    E, k, H, I = 256, 8, 256, 256
+    W = di.MoEWeights(2, E, H, I)
+    w13, w2 = W.materialize("cuda")
+    m = d.DAMoE(2000, k, E, H, I)
+    for T, alpha in [(2000, 0.05), (128, 0.2), (129, 10.0)]:
+        case = Case(T, T, E, k, H, I, alpha)
+        case.weights = W
+        out = m.fused_moe(case.x("cuda"), w13, w2, torch.from_numpy(case.ids).cuda(), torch.from_numpy(case.w).cuda(), 3)
+        meta = m.debug_fetch(T)
+        assert meta["status"] == 0
+        _check_route(meta, case, d.tile_ns())
+        _check_layer(out, case, tokens=list(range(0, T, max(1, T // 16))))
+    m.close()
+
+
 def test_edge_cases(d):
     case = config0(seed=3, T=5)
     t = _device_case(case)
