@@ -450,7 +450,7 @@ def run_ours(args):
     traffic = None
     if not fp8 and not is_trace:
         traffic = round(NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 * statistics.mean(c["active"] for c in rec_cells))
-    roofline = dict(bound="hbm", kernel=("gemm8" if fp8 else "gemm") + "_branch_kernel<0> (grouped gate/up GEMM + SwiGLU)", achieved=round(achieved, 1),
+    roofline = dict(bound="hbm", kernel=("gemm8_branch_kernel<0>" if fp8 else "gemm2_branch_kernel<0>") + " (grouped gate/up GEMM + SwiGLU, branching on the device-side variant id)", achieved=round(achieved, 1),
                     peak=pk["hbm_gbs"], unit="GB/s", frac=round(achieved / pk["hbm_gbs"], 4), traffic=traffic,
                     algorithmic_bytes=round(w13_bytes), peak_source=pk["source"], launch_ms=round(w13_ms, 4),
                     launches_timed=n_rec,
@@ -483,7 +483,8 @@ def run_ours(args):
                 vs_baseline=None, dtype="fp8" if fp8 else "bf16", data="synthetic", config=config,
                 aggregate_layers_per_s=round(world * 1e6 / us_per_layer, 2),
                 e2e=dict(value=round(e2e_us, 2), unit="us", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
-                gpu_launches=7 * steps, clocks=clocks, roofline=roofline, cpu_baseline=cpu, dispatch=dispatch,
+                gpu_launches=sum((1 if cells[i % len(cells)]["T"] * w["k"] <= 1024 else 3) + 4 for i in range(steps)),
+                clocks=clocks, roofline=roofline, cpu_baseline=cpu, dispatch=dispatch,
                 dispatch_overhead=overhead, device_status=status)
     print(json.dumps(line))
 
