@@ -54,6 +54,10 @@ TRACE_WORKLOAD = dict(name="kimi_k2_trace_500", E=384, k=8, H=7168, I=2048, T=40
 # scales, bf16 output; T in {16, 256, 4096} x alpha in {0.1, 1, 10}.
 FP8_WORKLOAD = dict(name="deepseek_v3_fp8_grid", E=256, k=8, H=7168, I=2048, T=4096, dtype="fp8",
                     grid=[(T, a) for T in (16, 256, 4096) for a in (0.1, 1.0, 10.0)], weight_seed=12345)
+# One expert-parallel shard (EP = 4) of the DeepSeek-V3 layer on one GPU: 64 local experts, routing
+# drawn over all 256 experts and masked to the shard; 200 batches, T log-uniform in [1, 2048].
+EP4_WORKLOAD = dict(name="deepseek_v3_ep4_shard_trace_200", E=64, E_global=256, k=8, H=7168, I=2048, T=2048,
+                    trace=(3000, 200), weight_seed=12345)
 # The same kind of trace on the headline shape (weights already resident): 48 batches, part of
 # the default line so that the dispatcher is also measured where token counts and skew vary.
 HEADLINE_TRACE = (2000, 48)
@@ -97,8 +101,11 @@ def make_cells(device, trace=None):
     cells = []
     for T, a, seed in specs:
         if True:
-            ids, wts, _ = di.routing_batch(seed, T, w["k"], w["E"], a)
-            hist = np.bincount(ids.reshape(-1), minlength=w["E"])
+            ids, wts, _ = di.routing_batch(seed, T, w["k"], w.get("E_global", w["E"]), a)
+            if "E_global" in w:
+                ids = di.shard_ids(ids, w["E"])
+            flat = ids.reshape(-1)
+            hist = np.bincount(flat[flat >= 0], minlength=w["E"])
             cell = dict(T=T, alpha=a, seed=seed, ids=ids, w=wts, active=int((hist > 0).sum()), hist=hist)
             if device is not None:
                 cell["x_host"] = di.activations(seed, T, w["H"]).pin_memory()
@@ -156,7 +163,7 @@ class ClockSampler:
 def layer_bytes_flops(cell, tile_n):
     """Algorithmic bytes and padded flops of one whole layer call (bf16)."""
     w = WORKLOAD
-    P = cell["T"] * w["k"]
+    P = int(cell["hist"].sum())          # valid (token, slot) pairs; fewer than T*k only for a masked shard
     A = cell["active"]
     eb = 1 if w.get("dtype") == "fp8" else 2
     wbytes = A * 3 * w["H"] * w["I"] * eb
@@ -170,7 +177,7 @@ def w13_launch_bytes(cell):
     """Algorithmic bytes of one gate/up GEMM launch: each activated expert's W13 once, the
     gathered activations read once, h written once."""
     w = WORKLOAD
-    P = cell["T"] * w["k"]
+    P = int(cell["hist"].sum())
     eb = 1 if w.get("dtype") == "fp8" else 2
     return cell["active"] * 2 * w["I"] * w["H"] * eb + P * w["H"] * eb + P * w["I"] * eb
 
@@ -468,7 +475,7 @@ def run_ours(args):
     mean_T = statistics.mean(c["T"] for c in cells)
     h2d = int(mean_T * w["H"] * 2 + 2 * mean_T * w["k"] * 4)
     d2h = int(mean_T * w["H"] * 2)
-    config = dict(workload=w["name"], E=w["E"], k=w["k"], H=w["H"], I=w["I"], T=w["T"] if not is_trace else "log-uniform [1, 4096]",
+    config = dict(workload=w["name"], E=w["E"], k=w["k"], H=w["H"], I=w["I"], T=w["T"] if not is_trace else f"log-uniform [1, {w['T']}]",
                   batches=len(cells), dispatch="auto/branch", table=table,
                   l2="inputs larger than L2: a step streams the activated experts' weights (GBs), never reused across steps",
                   parallelism="replicas only" if world > 1 else "single GPU")
@@ -496,7 +503,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="headline", choices=["headline", "small", "small_dense", "kimi_trace", "fp8_grid"],
+    ap.add_argument("--workload", default="headline", choices=["headline", "small", "small_dense", "kimi_trace", "fp8_grid", "ep4_trace"],
                     help="'small' is the reduced case used for ncu captures; 'kimi_trace' the 500-batch serving-trace stand-in")
     ap.add_argument("--no-table", action="store_true", help="ignore the committed tuning table")
     ap.add_argument("--table", default=None, help="tuning table file to load instead of the committed one")
@@ -504,7 +511,8 @@ def main():
     args = ap.parse_args()
     if args.workload != "headline":
         WORKLOAD.clear()
-        WORKLOAD.update(dict(small=SMALL_WORKLOAD, small_dense=SMALL_DENSE_WORKLOAD, kimi_trace=TRACE_WORKLOAD, fp8_grid=FP8_WORKLOAD)[args.workload])
+        WORKLOAD.update(dict(small=SMALL_WORKLOAD, small_dense=SMALL_DENSE_WORKLOAD, kimi_trace=TRACE_WORKLOAD, fp8_grid=FP8_WORKLOAD,
+                             ep4_trace=EP4_WORKLOAD)[args.workload])
     if args.impl == "reference":
         run_reference(args)
     else:

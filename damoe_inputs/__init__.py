@@ -228,6 +228,15 @@ def routing_batch(seed: int, T: int, k: int, E: int, alpha: float):
     return ids, w, np.exp(log_p)
 
 
+def shard_ids(ids: np.ndarray, E_local: int, shard: int = 0) -> np.ndarray:
+    """Expert-parallel view of a global routing: experts [shard*E_local, (shard+1)*E_local) are
+    renumbered from 0, every other id becomes -1 (the library skips ids outside [0, E))."""
+    lo = shard * E_local
+    out = ids.astype(np.int64) - lo
+    out[(out < 0) | (out >= E_local)] = -1
+    return out.astype(np.int32)
+
+
 def uniform_routing(seed: int, T: int, k: int, E: int):
     """Top-k of iid random logits: uniform routing without replacement (the
     'random inputs' a static per-bucket tuner profiles with, Section IV)."""

@@ -37,6 +37,9 @@ SHAPES = {
     "tiny": dict(E=8, k=2, H=1024, I=512),
     "dsv3": dict(E=256, k=8, H=7168, I=2048),
     "kimi": dict(E=384, k=8, H=7168, I=2048),
+    # one expert-parallel shard of the DeepSeek-V3 layer: 64 local experts of 256, routing drawn over
+    # all 256 and masked to the shard (the setting in which the paper measured its gains, EP = 4)
+    "dsv3_ep4": dict(E=64, k=8, H=7168, I=2048, E_global=256),
 }
 UNIFORM = "uniform"
 
@@ -186,10 +189,13 @@ def sweep(shape, buckets, alphas, seeds, reps, log_path, weight_seed=12345, devi
                     r = done[key]
                 else:
                     seed = 50000 + 977 * s + T            # tuning seeds, disjoint from evaluation seeds
+                    Eg = shape.get("E_global", E)
                     if alpha == UNIFORM:
-                        ids, wts = di.uniform_routing(seed, T, k, E)
+                        ids, wts = di.uniform_routing(seed, T, k, Eg)
                     else:
-                        ids, wts, _ = di.routing_batch(seed + int(round(alpha * 1000)), T, k, E, alpha)
+                        ids, wts, _ = di.routing_batch(seed + int(round(alpha * 1000)), T, k, Eg, alpha)
+                    if Eg != E:
+                        ids = di.shard_ids(ids, E)
                     x = di.activations(seed, T, H, device)
                     if fp8:
                         x, xs = di.quantize_e4m3_blocks(x, 1, 128)
@@ -201,7 +207,7 @@ def sweep(shape, buckets, alphas, seeds, reps, log_path, weight_seed=12345, devi
                     us = [time_call(lambda v=v: m.fused_moe(x, w13, w2, ids_d, w_d, v, out=out), reps) for v in range(VA)]
                     us += [1e9] * (V - VA)                   # variants not built for this dtype
                     meta = m.debug_fetch(T)
-                    hist = np.bincount(ids.reshape(-1), minlength=E)
+                    hist = np.bincount(ids.reshape(-1)[ids.reshape(-1) >= 0], minlength=E)
                     r = dict(T=T, alpha=alpha, seed=s, us=us, counts=hist.tolist(), active=int((hist > 0).sum()),
                              tiles=meta["tiles"].tolist(), status=meta["status"])
                     if log:

@@ -631,10 +631,11 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
   } else {
     // one persistent kernel per GEMM that branches on the variant id; when the CTA-pair variants
     // exist it is launched as clusters of two so that it can hold the whole family
-    if (c->pairs_ok) DAMOE_CUDA(c, launch_gemm2cta(0, -2, false, pack.m13, pack.ga, c->sm_count, st));
+    static const bool exp_1cta = getenv("DAMOE_EXP_BRANCH_1CTA") != nullptr;
+    if (c->pairs_ok && !exp_1cta) DAMOE_CUDA(c, launch_gemm2cta(0, -2, false, pack.m13, pack.ga, c->sm_count, st));
     else DAMOE_CUDA(c, launch_gemm(0, -1, false, pack.m13, pack.ga, c->sm_count, st));
     DAMOE_MARK(3);
-    if (c->pairs_ok) DAMOE_CUDA(c, launch_gemm2cta(1, -2, false, pack.m2, pack.ga, c->sm_count, st));
+    if (c->pairs_ok && !exp_1cta) DAMOE_CUDA(c, launch_gemm2cta(1, -2, false, pack.m2, pack.ga, c->sm_count, st));
     else DAMOE_CUDA(c, launch_gemm(1, -1, false, pack.m2, pack.ga, c->sm_count, st));
   }
   DAMOE_MARK(4);

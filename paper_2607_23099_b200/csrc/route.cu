@@ -19,6 +19,7 @@ namespace {
 constexpr int kScanThreads = 1024;
 constexpr int kWarpsPerRouteBlock = kPairsPerBlock / 32;
 constexpr int kMaxExemplars = 64;
+constexpr int kExPrefetchInts = 4096;  // exemplars of a bucket are staged in shared memory when they fit (16 KB)
 
 __global__ void __launch_bounds__(kPairsPerBlock) route_count_kernel(const int32_t* __restrict__ ids, int P, int E,
                                                                      int32_t* __restrict__ block_hist,
@@ -75,6 +76,47 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int* tot
 // thread per pair): it counts the histogram itself, and after the offsets are known ranks each
 // pair by brute force over the ids held in shared memory (rank = earlier pairs with the same
 // expert), which gives the same canonical stable order as the three-kernel path.
+// Exclusive scans of NV ints per thread at once (one set of block-wide synchronisations for
+// all of them); total[v] gets each sum.  s_warp must hold NV * 33 ints.
+template <int NV>
+__device__ __forceinline__ void block_exclusive_scan_vec(const int (&v)[NV], int (&ex)[NV], int (&total)[NV],
+                                                         int* s_warp) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc[NV];
+#pragma unroll
+  for (int q = 0; q < NV; ++q) {
+    inc[q] = v[q];
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int o = __shfl_up_sync(0xffffffffu, inc[q], d);
+      if (lane >= d) inc[q] += o;
+    }
+  }
+  __syncthreads();
+  if (lane == 31) {
+#pragma unroll
+    for (int q = 0; q < NV; ++q) s_warp[q * 33 + warp] = inc[q];
+  }
+  __syncthreads();
+  if (warp < NV) {  // warp q scans the 32 warp totals of quantity q
+    const int w = s_warp[warp * 33 + lane];
+    int winc = w;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int o = __shfl_up_sync(0xffffffffu, winc, d);
+      if (lane >= d) winc += o;
+    }
+    s_warp[warp * 33 + lane] = winc - w;
+    if (lane == 31) s_warp[warp * 33 + 32] = winc;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < NV; ++q) {
+    total[q] = s_warp[q * 33 + 32];
+    ex[q] = s_warp[q * 33 + warp] + inc[q] - v[q];
+  }
+}
+
 template <bool FUSED>
 __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __restrict__ block_hist, int nblocks, int E,
                                                                   Workspace ws, SelectorArgs sel,
@@ -85,18 +127,34 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
   __shared__ int s_hist[kMaxE];
   __shared__ int s_ids[FUSED ? kScanThreads : 1];
   __shared__ int s_offs[FUSED ? kMaxE : 1];
+  // the bucket's table entries, copied in before the wait on the preceding kernel: they are
+  // constants of the loaded table, so fetching them overlaps that kernel's tail
+  __shared__ int s_ex[kExPrefetchInts];
+  __shared__ int s_exv[kMaxExemplars];
+  __shared__ long long s_cost[4 * kNumVariants];
+  __shared__ long long s_costv[kNumVariants];
   __shared__ int s_sorted[kMaxE];
-  __shared__ int s_warp[33];
+  __shared__ int s_warp[(kNumVariants + 2) * 33];
+  __shared__ int s_rank[kMaxE];
   __shared__ unsigned long long s_red[2][32];
   __shared__ int s_tiles[kNumVariants];
   __shared__ long long s_score[kMaxExemplars];
   __shared__ int s_active;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   pdl_launch_dependents();
+  const bool select = !stats_only && sel.forced < 0;
+  const bool ex_staged = select && sel.mode == DAMOE_MODE_EXEMPLAR && sel.n_exemplars * E <= kExPrefetchInts;
+  if (select && sel.mode == DAMOE_MODE_EXEMPLAR) {
+    if (ex_staged)
+      for (int i = tid; i < sel.n_exemplars * E; i += kScanThreads) s_ex[i] = sel.exemplars[i];
+    if (tid < sel.n_exemplars) s_exv[tid] = sel.ex_variant[tid];
+  } else if (select && sel.mode == DAMOE_MODE_COST) {
+    if (tid < 4 * kNumVariants) s_cost[tid] = sel.cost[tid];
+  }
   if (FUSED) {
     for (int e = tid; e < E; e += kScanThreads) s_hist[e] = 0;
-    __syncthreads();
   }
+  __syncthreads();
   pdl_wait();
 
   if (FUSED) {
@@ -164,14 +222,37 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
   __syncthreads();
 
   const int t_e = (tid < E) ? s_hist[tid] : 0;
-  int total;
-  // offsets
+  // one block scan for everything: offsets (t_e), active experts (t_e > 0) and, per variant,
+  // the token tiles ceil(t_e / N_v)
   {
-    const int ex = block_exclusive_scan(t_e, s_warp, &total);
-    if (tid < E) ws.offsets[tid] = ex;
-    if (tid == 0) ws.offsets[E] = total;
+    constexpr int NV = kNumVariants + 2;
+    int val[NV], ex[NV], tot[NV];
+    val[0] = t_e;
+    val[1] = t_e > 0 ? 1 : 0;
+#pragma unroll
+    for (int v = 0; v < kNumVariants; ++v) {
+      const int n = variant_desc(v).tile_n;
+      val[2 + v] = (t_e + n - 1) / n;
+    }
+    block_exclusive_scan_vec<NV>(val, ex, tot, s_warp);
+    if (tid < E) {
+      ws.offsets[tid] = ex[0];
+#pragma unroll
+      for (int v = 0; v < kNumVariants; ++v) ws.ntile_prefix[v * (E + 1) + tid] = ex[2 + v];
+    }
+    if (tid == 0) {
+      ws.offsets[E] = tot[0];
+      s_active = tot[1];
+      *ws.active = tot[1];
+#pragma unroll
+      for (int v = 0; v < kNumVariants; ++v) {
+        ws.ntile_prefix[v * (E + 1) + E] = tot[2 + v];
+        ws.tiles[v] = tot[2 + v];
+        s_tiles[v] = tot[2 + v];
+      }
+    }
     if (FUSED) {
-      if (tid < E) s_offs[tid] = ex;
+      if (tid < E) s_offs[tid] = ex[0];
       __syncthreads();
       const int e = s_ids[tid];
       if (e >= 0) {
@@ -184,26 +265,7 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
       } else if (tid < P) {
         ws.inv[tid] = -1;
       }
-      if (tid < P && tid >= total) ws.perm[tid] = -1;  // sorted positions past the valid count
-    }
-  }
-  // active experts
-  {
-    block_exclusive_scan(t_e > 0 ? 1 : 0, s_warp, &total);
-    if (tid == 0) {
-      s_active = total;
-      *ws.active = total;
-    }
-  }
-  // token tiles per variant: exclusive scan of ceil(t_e / N_v)
-  for (int v = 0; v < kNumVariants; ++v) {
-    const int n = variant_desc(v).tile_n;
-    const int ex = block_exclusive_scan((t_e + n - 1) / n, s_warp, &total);
-    if (tid < E) ws.ntile_prefix[v * (E + 1) + tid] = ex;
-    if (tid == 0) {
-      ws.ntile_prefix[v * (E + 1) + E] = total;
-      ws.tiles[v] = total;
-      s_tiles[v] = total;
+      if (tid < P && tid >= tot[0]) ws.perm[tid] = -1;  // sorted positions past the valid count
     }
   }
   __syncthreads();
@@ -218,20 +280,52 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
   }
   int chosen = 0;
   if (sel.mode == DAMOE_MODE_EXEMPLAR) {
-    // descending sort by rank counting: rank_i = #{j : t_j > t_i or (t_j == t_i and j < i)}
-    if (tid < E) {
-      int rank = 0;
-      for (int j = 0; j < E; ++j) {
-        const int tj = s_hist[j];
-        rank += (tj > t_e) || (tj == t_e && j < tid);
+    // Descending sort of the histogram (values only: equal counts are interchangeable).
+    if (P < kScanThreads) {
+      // Small batch: counts are below 1024, so sort by counting.  s_rank[c] = experts with count
+      // 1023 - c (descending order of c = ascending index), scanned to start positions.
+      s_rank[tid] = 0;
+      __syncthreads();
+      if (tid < E) atomicAdd(&s_rank[kScanThreads - 1 - t_e], 1);
+      __syncthreads();
+      int start, tot1;
+      start = block_exclusive_scan(s_rank[tid], s_warp, &tot1);
+      __syncthreads();
+      s_rank[tid] = start;
+      __syncthreads();
+      if (tid < E) s_sorted[atomicAdd(&s_rank[kScanThreads - 1 - t_e], 1)] = t_e;
+      __syncthreads();
+    } else {
+      // rank counting: rank_i = #{j : t_j > t_i or (t_j == t_i and j < i)}.  Consecutive lanes own
+      // consecutive experts i and walk the same j (shared-memory broadcasts, no bank
+      // conflicts); the j range is split over R groups of warps whose partial counts meet in a
+      // shared-memory atomic.
+      int e_pow2 = 32;
+      while (e_pow2 < E) e_pow2 <<= 1;
+      const int R = kScanThreads / e_pow2;           // >= 1 because E <= 1024
+      for (int i = tid; i < E; i += kScanThreads) s_rank[i] = 0;
+      __syncthreads();
+      {
+        const int i = tid % e_pow2, r = tid / e_pow2;
+        if (i < E && r < R) {
+          const int ti = s_hist[i];
+          const int j0 = (E * r) / R, j1 = (E * (r + 1)) / R;
+          int cnt = 0;
+          for (int j = j0; j < j1; ++j) {
+            const int tj = s_hist[j];
+            cnt += (tj > ti) | ((tj == ti) & (j < i));
+          }
+          atomicAdd(&s_rank[i], cnt);
+        }
       }
-      s_sorted[rank] = t_e;
+      __syncthreads();
+      if (tid < E) s_sorted[s_rank[tid]] = s_hist[tid];
+      __syncthreads();
     }
-    __syncthreads();
     // one warp per exemplar: exact integer dot product with the Q30 unit vector
     for (int m = warp; m < sel.n_exemplars; m += kScanThreads / 32) {
       long long acc = 0;
-      const int32_t* ex = sel.exemplars + static_cast<size_t>(m) * E;
+      const int32_t* ex = ex_staged ? s_ex + m * E : sel.exemplars + static_cast<size_t>(m) * E;
       for (int i = lane; i < E; i += 32) acc += static_cast<long long>(s_sorted[i]) * static_cast<long long>(ex[i]);
 #pragma unroll
       for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, d);
@@ -242,7 +336,7 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
       int best = 0;
       for (int m = 1; m < sel.n_exemplars; ++m)
         if (s_score[m] > s_score[best]) best = m;
-      chosen = sel.ex_variant[best];
+      chosen = s_exv[best];
     }
   } else if (sel.mode == DAMOE_MODE_EFFEXP_BINS) {
     if (tid == 0) {
@@ -253,19 +347,18 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
       chosen = sel.bin_variant[r];
     }
   } else {  // DAMOE_MODE_COST
-    if (tid == 0) {
+    if (tid < kNumVariants) {
+      const int v = tid;
       const long long A = s_active;
-      long long best_cost = 0;
-      for (int v = 0; v < kNumVariants; ++v) {
-        const long long tiles = s_tiles[v];
-        const long long mem = sel.cost[1 * kNumVariants + v] * A + sel.cost[2 * kNumVariants + v] * (tiles - A);
-        const long long mma = sel.cost[3 * kNumVariants + v] * tiles * variant_desc(v).tile_n;
-        const long long c = sel.cost[0 * kNumVariants + v] + (mem > mma ? mem : mma);
-        if (v == 0 || c < best_cost) {
-          best_cost = c;
-          chosen = v;
-        }
-      }
+      const long long tiles = s_tiles[v];
+      const long long mem = s_cost[1 * kNumVariants + v] * A + s_cost[2 * kNumVariants + v] * (tiles - A);
+      const long long mma = s_cost[3 * kNumVariants + v] * tiles * variant_desc(v).tile_n;
+      s_costv[v] = s_cost[0 * kNumVariants + v] + (mem > mma ? mem : mma);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      for (int v = 1; v < kNumVariants; ++v)
+        if (s_costv[v] < s_costv[chosen]) chosen = v;
     }
   }
   if (tid == 0) {
