@@ -253,6 +253,28 @@ def geomean(xs):
     return math.exp(sum(math.log(x) for x in xs) / len(xs))
 
 
+def retime_auto(m, d, cells, run, rows, reps=3):
+    """AUTO re-timed under the selection mode currently set, against the STATIC / best times of
+    ``rows`` (from compare_dispatch on the same batches)."""
+    stream = torch.cuda.current_stream()
+    ratios, gaps = [], []
+    for c, r in zip(cells, rows):
+        run(c, d.VARIANT_AUTO)
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            run(c, d.VARIANT_AUTO)
+            b.record(stream)
+            b.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3)
+        t = statistics.median(ts)
+        ratios.append(r["static_us"] / t)
+        gaps.append(t / r["best_us"])
+    return dict(geomean_speedup_vs_static=round(geomean(ratios), 4), peak_speedup_vs_static=round(max(ratios), 4),
+                geomean_gap_to_best=round(geomean(gaps), 4))
+
+
 def compare_dispatch(m, d, cells, run, pk, reps=3):
     """Per batch: AUTO vs STATIC vs every variant (median of reps), roofline of the chosen one."""
     ns = d.tile_ns()
@@ -434,6 +456,16 @@ def run_ours(args):
     # ---- adaptive vs static vs per-batch best ----
     summary, rows = compare_dispatch(m, d, cells, run, pk)
     dispatch = dict(summary, table=table, cells=rows if len(rows) <= 64 else rows[:64])
+    if table != "built-in cost model":
+        # the same table under the other two selection modes (its header's mode was used above)
+        dispatch["selector_mode"] = "table default (Effective-Experts bins)"
+        for name, mode in (("exemplar", d.MODE_EXEMPLAR), ("cost", d.MODE_COST)):
+            try:
+                m.set_selector_mode(mode)
+                dispatch["auto_" + name] = retime_auto(m, d, cells, run, rows)
+            except d.DamoeError:
+                pass
+        m.set_selector_mode(d.MODE_EFFEXP_BINS)
     if not is_trace and args.workload == "headline":
         tcells = make_cells(device, trace=HEADLINE_TRACE)
         tsum, trows = compare_dispatch(m, d, tcells, run, pk)

@@ -183,6 +183,15 @@ int damoe_set_fp8_scales(damoe_ctx* ctx, const float* x_scale, const float* w13_
  */
 int damoe_load_tuning_table(damoe_ctx* ctx, const void* bytes, size_t nbytes);
 
+/*
+ * Override the selection mode of the loaded table (DAMOE_MODE_EXEMPLAR: the paper's sorted-
+ * histogram cosine match, Section IV-B; DAMOE_MODE_EFFEXP_BINS: thresholds on Effective
+ * Experts; DAMOE_MODE_COST: integer cost model over padded tiles and weight reloads).  A table
+ * written by the auto-tuner carries the data of all three; the mode in its header is only the
+ * default.  DAMOE_ERR_INVALID_ARG when no table is loaded or a bucket lacks that mode's data.
+ */
+int damoe_set_selector_mode(damoe_ctx* ctx, int mode);
+
 /* Select how DAMOE_VARIANT_AUTO dispatches (default DAMOE_DISPATCH_BRANCH). */
 int damoe_set_dispatch(damoe_ctx* ctx, int dispatch_mode);
 

@@ -26,7 +26,7 @@ EXPORTS = [
     "damoe_create", "damoe_destroy", "damoe_last_error", "damoe_route_stats", "damoe_fused_moe",
     "damoe_fused_moe_host", "damoe_set_fp8_scales", "damoe_load_tuning_table", "damoe_set_dispatch",
     "damoe_variant_count", "damoe_variant_info", "damoe_debug_fetch", "damoe_dispatch_microbench",
-    "damoe_set_profiling", "damoe_get_stage_ms", "damoe_route_stats_noalloc",
+    "damoe_set_profiling", "damoe_get_stage_ms", "damoe_route_stats_noalloc", "damoe_set_selector_mode",
 ]
 
 
@@ -47,6 +47,7 @@ def _load() -> ctypes.CDLL:
     lib.damoe_set_fp8_scales.argtypes = [vp, vp, vp, vp]
     lib.damoe_load_tuning_table.argtypes = [vp, ctypes.c_char_p, ctypes.c_size_t]
     lib.damoe_set_dispatch.argtypes = [vp, i32]
+    lib.damoe_set_selector_mode.argtypes = [vp, i32]
     lib.damoe_variant_count.argtypes = []
     lib.damoe_variant_info.argtypes = [i32] + [ctypes.POINTER(i32)] * 4
     lib.damoe_debug_fetch.argtypes = [vp] * 7
@@ -175,6 +176,9 @@ class DAMoE:
 
     def load_tuning_table(self, blob: bytes):
         self._check(_lib.damoe_load_tuning_table(self._ctx, blob, len(blob)))
+
+    def set_selector_mode(self, mode: int):
+        self._check(_lib.damoe_set_selector_mode(self._ctx, mode))
 
     def set_dispatch(self, mode: int):
         self._check(_lib.damoe_set_dispatch(self._ctx, mode))

@@ -460,6 +460,18 @@ int damoe_set_dispatch(damoe_ctx* c, int mode) {
   return DAMOE_OK;
 }
 
+int damoe_set_selector_mode(damoe_ctx* c, int mode) {
+  if (!c) return DAMOE_ERR_INVALID_ARG;
+  if (!c->has_table) return fail(c, DAMOE_ERR_INVALID_ARG, "no tuning table is loaded");
+  if (mode < DAMOE_MODE_EXEMPLAR || mode > DAMOE_MODE_COST) return fail(c, DAMOE_ERR_INVALID_ARG, "mode %d", mode);
+  for (const TableBucket& b : c->buckets) {
+    if (mode == DAMOE_MODE_EXEMPLAR && b.n_ex == 0) return fail(c, DAMOE_ERR_INVALID_ARG, "bucket T=%d has no exemplar", b.T);
+    if (mode == DAMOE_MODE_EFFEXP_BINS && b.n_bins == 0) return fail(c, DAMOE_ERR_INVALID_ARG, "bucket T=%d has no bin", b.T);
+  }
+  c->table_mode = mode;
+  return DAMOE_OK;
+}
+
 int damoe_set_fp8_scales(damoe_ctx* c, const float* x_scale, const float* w13_scale, const float* w2_scale) {
   if (!c) return DAMOE_ERR_INVALID_ARG;
   if (c->dtype != DAMOE_FP8_E4M3_BLOCK128) return fail(c, DAMOE_ERR_INVALID_ARG, "context is not FP8");

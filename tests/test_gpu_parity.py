@@ -203,6 +203,15 @@ def test_selected_variant_matches_oracle_given_the_same_table(d):
                 assert meta["variant_id"] == want and meta["status"] == 0
                 seen.add(want)
         assert len(seen) >= 2
+    # the table's mode is only a default: switch the loaded table between modes
+    table = _table_for(E, k, [16, 128, 512], d.MODE_EXEMPLAR, V, ns)
+    m.load_tuning_table(tuning.pack_table(table, E, k, H, I, d.BF16, V))
+    ids, w, _ = di.routing_batch(77, 100, k, E, 0.3)
+    x = di.activations(77, 100, H, "cuda")
+    for mode in (d.MODE_COST, d.MODE_EFFEXP_BINS, d.MODE_EXEMPLAR):
+        m.set_selector_mode(mode)
+        m.fused_moe(x, w13, w2, torch.from_numpy(ids).cuda(), torch.from_numpy(w).cuda(), d.VARIANT_AUTO)
+        assert m.debug_fetch(100)["variant_id"] == route.select_variant(dict(table, mode=mode), route.histogram(ids, E), 100, ns)
     # malformed / mismatched tables are refused
     good = tuning.pack_table(_table_for(E, k, [16], d.MODE_COST, V, ns), E, k, H, I, d.BF16, V)
     with pytest.raises(d.DamoeError) as ei:
