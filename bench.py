@@ -48,6 +48,7 @@ SMALL_WORKLOAD = dict(name="profile_small_E32_T8", E=32, k=8, H=7168, I=2048, T=
 # the full shape) on 16 experts, 1.4 GB of weights.  Only for ncu captures.
 SMALL_DENSE_WORKLOAD = dict(name="profile_small_dense_E16_T512", E=16, k=8, H=7168, I=2048, T=512,
                             alphas=[10.0], seeds=[0, 1], weight_seed=12345)
+SMALL_DENSE_FP8_WORKLOAD = dict(SMALL_DENSE_WORKLOAD, name="profile_small_dense_fp8_E16_T512", dtype="fp8")
 TRACE_WORKLOAD = dict(name="kimi_k2_trace_500", E=384, k=8, H=7168, I=2048, T=4096, trace=(1000, 500),
                       weight_seed=12345)
 # FP8 configuration: E4M3 weights with 128x128 block scales, E4M3 activations with 1x128 group
@@ -535,7 +536,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="headline", choices=["headline", "small", "small_dense", "kimi_trace", "fp8_grid", "ep4_trace"],
+    ap.add_argument("--workload", default="headline", choices=["headline", "small", "small_dense", "small_dense_fp8", "kimi_trace", "fp8_grid", "ep4_trace"],
                     help="'small' is the reduced case used for ncu captures; 'kimi_trace' the 500-batch serving-trace stand-in")
     ap.add_argument("--no-table", action="store_true", help="ignore the committed tuning table")
     ap.add_argument("--table", default=None, help="tuning table file to load instead of the committed one")
@@ -543,7 +544,8 @@ def main():
     args = ap.parse_args()
     if args.workload != "headline":
         WORKLOAD.clear()
-        WORKLOAD.update(dict(small=SMALL_WORKLOAD, small_dense=SMALL_DENSE_WORKLOAD, kimi_trace=TRACE_WORKLOAD, fp8_grid=FP8_WORKLOAD,
+        WORKLOAD.update(dict(small=SMALL_WORKLOAD, small_dense=SMALL_DENSE_WORKLOAD, small_dense_fp8=SMALL_DENSE_FP8_WORKLOAD,
+                             kimi_trace=TRACE_WORKLOAD, fp8_grid=FP8_WORKLOAD,
                              ep4_trace=EP4_WORKLOAD)[args.workload])
     if args.impl == "reference":
         run_reference(args)

@@ -249,24 +249,38 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
         }
         tc_fence_after();
         const uint32_t t0 = tmem_base + (lane_base << 16) + pb * C::kAccCols + col0;
-        // only the 16-column (8 for the narrowest tile) chunks that hold valid tokens are promoted
+        // Only the 16-column (8 for the narrowest tile) chunks that hold valid tokens are promoted.
+        // All TMEM loads of a group of up to 32 columns (gate and up) are issued before the one
+        // wait, so their latency is paid once per group instead of once per chunk.
         constexpr int CH = CW < 16 ? CW : 16;
+        constexpr int GW = CW < 32 ? CW : 32;   // columns per group
 #pragma unroll
-        for (int c = 0; c < CW; c += CH) {
-          if (col0 + c < item.valid) {  // warp-uniform
-            float p[CH];
-            tmem_ld_cols<CH>(t0 + c, p);
+        for (int g0 = 0; g0 < CW; g0 += GW) {
+          if (col0 + g0 < item.valid) {  // warp-uniform
+            uint32_t pg[GW], pu[(KIND == 0) ? GW : 1];
 #pragma unroll
-            for (int j = 0; j < CH; ++j) {
-              const float sx = __shfl_sync(0xffffffffu, (c + j < 32) ? sx0 : sx1, (c + j) & 31);
-              acc_g[c + j] = fmaf(p[j], sx * swg, acc_g[c + j]);
+            for (int c = 0; c < GW; c += CH) {
+              if (col0 + g0 + c < item.valid) {
+                if constexpr (CH == 8) {
+                  tmem_ld_x8(t0 + g0 + c, *reinterpret_cast<uint32_t(*)[8]>(&pg[c]));
+                  if constexpr (KIND == 0) tmem_ld_x8(t0 + BN + g0 + c, *reinterpret_cast<uint32_t(*)[8]>(&pu[c]));
+                } else {
+                  tmem_ld_x16(t0 + g0 + c, *reinterpret_cast<uint32_t(*)[16]>(&pg[c]));
+                  if constexpr (KIND == 0) tmem_ld_x16(t0 + BN + g0 + c, *reinterpret_cast<uint32_t(*)[16]>(&pu[c]));
+                }
+              }
             }
-            if (KIND == 0) {
-              tmem_ld_cols<CH>(t0 + BN + c, p);
+            tmem_ld_wait();
 #pragma unroll
-              for (int j = 0; j < CH; ++j) {
-                const float sx = __shfl_sync(0xffffffffu, (c + j < 32) ? sx0 : sx1, (c + j) & 31);
-                acc_u[c + j] = fmaf(p[j], sx * swu, acc_u[c + j]);
+            for (int c = 0; c < GW; c += CH) {
+              if (col0 + g0 + c < item.valid) {
+#pragma unroll
+                for (int j = 0; j < CH; ++j) {
+                  const int col = g0 + c + j;
+                  const float sx = __shfl_sync(0xffffffffu, (col < 32) ? sx0 : sx1, col & 31);
+                  acc_g[col] = fmaf(__uint_as_float(pg[c + j]), sx * swg, acc_g[col]);
+                  if constexpr (KIND == 0) acc_u[col] = fmaf(__uint_as_float(pu[c + j]), sx * swu, acc_u[col]);
+                }
               }
             }
           }
