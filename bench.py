@@ -72,7 +72,7 @@ def table_path(w):
 # activated experts of the captured cell (profiles/gemm_gate_up_small_E32_T8_ncu_full.md):
 # bytes per activated expert.  The capture is of the reduced case; traffic grows in proportion
 # to the activated experts, so bench scales it by its own cells' counts.
-NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 = 59.05e6
+NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 = 59.01e6
 
 
 def peaks():
