@@ -48,6 +48,9 @@ SMALL_WORKLOAD = dict(name="profile_small_E32_T8", E=32, k=8, H=7168, I=2048, T=
 # the full shape) on 16 experts, 1.4 GB of weights.  Only for ncu captures.
 SMALL_DENSE_WORKLOAD = dict(name="profile_small_dense_E16_T512", E=16, k=8, H=7168, I=2048, T=512,
                             alphas=[10.0], seeds=[0, 1], weight_seed=12345)
+# The same regime with enough work items for several waves on every variant (2.8 GB of weights).
+MID_DENSE_WORKLOAD = dict(name="profile_mid_dense_E32_T1024", E=32, k=8, H=7168, I=2048, T=1024,
+                          alphas=[10.0], seeds=[0, 1], weight_seed=12345)
 SMALL_DENSE_FP8_WORKLOAD = dict(SMALL_DENSE_WORKLOAD, name="profile_small_dense_fp8_E16_T512", dtype="fp8")
 TRACE_WORKLOAD = dict(name="kimi_k2_trace_500", E=384, k=8, H=7168, I=2048, T=4096, trace=(1000, 500),
                       weight_seed=12345)
@@ -169,8 +172,14 @@ def layer_bytes_flops(cell, tile_n):
     eb = 1 if w.get("dtype") == "fp8" else 2
     wbytes = A * 3 * w["H"] * w["I"] * eb
     act = P * w["H"] * eb * 2 + P * w["I"] * eb * 2 + P * w["H"] * 4 * 2 + cell["T"] * w["H"] * (eb + 2) + 16 * P
-    # full tiles cost tile_n columns; the ragged last tile of an expert issues MMAs of ceil16(rest) columns
-    padded_cols = int(sum((int(t) // tile_n) * tile_n + (-(-(int(t) % tile_n) // 16) * 16) for t in cell["hist"]))
+    # an expert's t tokens are split evenly over ceil(t / tile_n) tiles; each tile issues MMAs of ceil16(size) columns
+    def cols(t):
+        if t == 0:
+            return 0
+        nt = -(-t // tile_n)
+        base, rem = divmod(t, nt)
+        return rem * (-(-(base + 1) // 16) * 16) + (nt - rem) * (-(-base // 16) * 16)
+    padded_cols = int(sum(cols(int(t)) for t in cell["hist"]))
     return wbytes + act, padded_cols * 6 * w["H"] * w["I"], P * 6 * w["H"] * w["I"]
 
 
@@ -536,7 +545,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="headline", choices=["headline", "small", "small_dense", "small_dense_fp8", "kimi_trace", "fp8_grid", "ep4_trace"],
+    ap.add_argument("--workload", default="headline", choices=["headline", "small", "small_dense", "mid_dense", "small_dense_fp8", "kimi_trace", "fp8_grid", "ep4_trace"],
                     help="'small' is the reduced case used for ncu captures; 'kimi_trace' the 500-batch serving-trace stand-in")
     ap.add_argument("--no-table", action="store_true", help="ignore the committed tuning table")
     ap.add_argument("--table", default=None, help="tuning table file to load instead of the committed one")
@@ -544,7 +553,7 @@ def main():
     args = ap.parse_args()
     if args.workload != "headline":
         WORKLOAD.clear()
-        WORKLOAD.update(dict(small=SMALL_WORKLOAD, small_dense=SMALL_DENSE_WORKLOAD, small_dense_fp8=SMALL_DENSE_FP8_WORKLOAD,
+        WORKLOAD.update(dict(small=SMALL_WORKLOAD, small_dense=SMALL_DENSE_WORKLOAD, mid_dense=MID_DENSE_WORKLOAD, small_dense_fp8=SMALL_DENSE_FP8_WORKLOAD,
                              kimi_trace=TRACE_WORKLOAD, fp8_grid=FP8_WORKLOAD,
                              ep4_trace=EP4_WORKLOAD)[args.workload])
     if args.impl == "reference":

@@ -41,7 +41,12 @@ struct damoe_ctx {
   const float* w13_scale = nullptr;
   const float* w2_scale = nullptr;
   bool pairs_ok = false;  // CTA-pair variants need an even number of 128-row weight tiles in both GEMMs
-  int num_variants() const { return dtype != DAMOE_BF16 ? kNumVariantsFp8 : pairs_ok ? kNumVariants : kNumVariants1Cta; }
+  // which ids of the family this context can run: fp8 has ids 0..3; bf16 all but, possibly, the pairs
+  bool variant_ok(int v) const {
+    if (v < 0 || v >= kNumVariants) return false;
+    if (dtype != DAMOE_BF16) return v < kNumVariantsFp8;
+    return pairs_ok || !variant_is_pair(v);
+  }
   // staging for the host-buffer entry point
   void *st_x = nullptr, *st_ids = nullptr, *st_w = nullptr, *st_out = nullptr;
   // DAMOE_DISPATCH_GRAPH_SWITCH: the last layer call as a graph with a conditional SWITCH node
@@ -131,7 +136,7 @@ void default_cost_model(const damoe_ctx* c, int64_t* cost) {
     cost[1 * kNumVariants + v] = static_cast<int64_t>(wbytes / 6.5e12 * 1e12);
     cost[2 * kNumVariants + v] = static_cast<int64_t>(wbytes / 13e12 * 1e12);
     cost[3 * kNumVariants + v] = static_cast<int64_t>(flops_col / (1.4e15 * eff) * 1e12);
-    if (v >= c->num_variants()) cost[0 * kNumVariants + v] = 1ll << 36;  // not built for this dtype: never chosen
+    if (!c->variant_ok(v)) cost[0 * kNumVariants + v] = 1ll << 36;  // this context cannot run it: never chosen
   }
 }
 
@@ -224,6 +229,8 @@ void build_pack(const damoe_ctx* c, LaunchPack* p) {
   ga.h = c->ws.h;
   ga.y = c->ws.y;
   ga.E = c->E; ga.H = c->H; ga.I = c->I;
+  static const int even = getenv("DAMOE_EVEN_SPLIT") ? atoi(getenv("DAMOE_EVEN_SPLIT")) : 1;
+  ga.even_split = even;
   p->ga = ga;
   GemmArgs8 g13{}, g2{};
   g13.ntile_prefix = g2.ntile_prefix = c->ws.ntile_prefix;
@@ -235,6 +242,7 @@ void build_pack(const damoe_ctx* c, LaunchPack* p) {
   g13.hs_T = g2.hs_T = c->ws.hs_T;
   g13.y = g2.y = c->ws.y;
   g13.E = g2.E = c->E; g13.H = g2.H = c->H; g13.I = g2.I = c->I; g13.max_P = g2.max_P = c->max_P;
+  g13.even_split = g2.even_split = even;
   g13.w_scale = c->w13_scale; g13.act_scale_T = c->ws.xs_T;
   g2.w_scale = c->w2_scale; g2.act_scale_T = c->ws.hs_T;
   p->g13 = g13;
@@ -245,7 +253,7 @@ void build_pack(const damoe_ctx* c, LaunchPack* p) {
 cudaError_t enqueue_gemm(const damoe_ctx* c, const LaunchPack& p, int kind, int v, bool predicated, cudaStream_t st) {
   const GemmMaps& maps = kind == 0 ? p.m13 : p.m2;
   if (c->dtype != DAMOE_BF16) return launch_gemm8(kind, v, predicated, maps, kind == 0 ? p.g13 : p.g2, c->sm_count, st);
-  if (v >= kNumVariants1Cta) return launch_gemm2cta(kind, v, predicated, maps, p.ga, c->sm_count, st);
+  if (variant_is_pair(v)) return launch_gemm2cta(kind, v, predicated, maps, p.ga, c->sm_count, st);
   return launch_gemm(kind, v, predicated, maps, p.ga, c->sm_count, st);
 }
 
@@ -299,7 +307,7 @@ int graph_switch_call(damoe_ctx* c, const void* x, const int32_t* ids, const flo
     if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess)
       return fail(c, DAMOE_ERR_CUDA, "capturing the head of the dispatch graph failed");
     // the SWITCH node: body v = both GEMMs of variant v
-    const int nv = c->num_variants();
+    const int nv = kNumVariants;
     cudaGraphNodeParams cp{};
     cp.type = cudaGraphNodeTypeConditional;
     cp.conditional.handle = handle;
@@ -308,6 +316,7 @@ int graph_switch_call(damoe_ctx* c, const void* x, const int32_t* ids, const flo
     cudaGraphNode_t cond;
     DAMOE_CUDA(c, cudaGraphAddNode(&cond, g, head.data(), head.size(), &cp));
     for (int v = 0; v < nv; ++v) {
+      if (!c->variant_ok(v)) continue;  // never selected on this context: its body stays empty
       DAMOE_CUDA(c, cudaStreamBeginCaptureToGraph(cs, cp.conditional.phGraph_out[v], nullptr, nullptr, 0, mode));
       cudaError_t a = enqueue_gemm(c, pack, 0, v, false, cs);
       cudaError_t b = enqueue_gemm(c, pack, 1, v, false, cs);
@@ -424,14 +433,10 @@ int damoe_create(damoe_ctx** out, int device, int max_T, int k, int E, int H, in
   default_cost_model(c, cost);
   if (cudaMemcpy(c->default_cost, cost, sizeof(cost), cudaMemcpyHostToDevice) != cudaSuccess) return bail(DAMOE_ERR_CUDA);
 
-  for (int v = 0; v < c->num_variants(); ++v) {
+  for (int v = 0; v < kNumVariants; ++v) {
     const uint32_t n = variant_desc(v).tile_n;
     if (make_map(c, &c->map_x[v], c->ws.x_perm, P, H, n) != DAMOE_OK) return bail(DAMOE_ERR_CUDA);
     if (make_map(c, &c->map_h[v], c->ws.h, P, I, n) != DAMOE_OK) return bail(DAMOE_ERR_CUDA);
-  }
-  for (int v = c->num_variants(); v < kNumVariants; ++v) {
-    c->map_x[v] = c->map_x[0];
-    c->map_h[v] = c->map_h[0];
   }
   *out = c;
   return DAMOE_OK;
@@ -503,7 +508,7 @@ int damoe_load_tuning_table(damoe_ctx* c, const void* bytes, size_t nbytes) {
     if (n) memcpy(blob.data() + o, src, n);
     return o;
   };
-  auto bad_variant = [&](int32_t v) { return v < 0 || v >= c->num_variants(); };
+  auto bad_variant = [&](int32_t v) { return !c->variant_ok(v); };
   for (uint32_t i = 0; i < nb; ++i) {
     TableBucket& b = buckets[i];
     b.T = (int)r.get<uint32_t>();
@@ -539,7 +544,8 @@ int damoe_load_tuning_table(damoe_ctx* c, const void* bytes, size_t nbytes) {
     if (!r.ok) return fail(c, DAMOE_ERR_TABLE_FORMAT, "truncated bucket %u", i);
     for (int t = 0; t < 4 * kNumVariants; ++t)
       if (cost[t] < 0 || cost[t] > (1ll << 36)) return fail(c, DAMOE_ERR_TABLE_FORMAT, "cost out of range in bucket %u", i);
-    for (int v = c->num_variants(); v < kNumVariants; ++v) cost[v] = 1ll << 36;  // variants not built for this dtype
+    for (int v = 0; v < kNumVariants; ++v)
+      if (!c->variant_ok(v)) cost[v] = 1ll << 36;  // variants this context cannot run
     b.off_ex = put(ex.data(), ex.size() * 4);
     b.off_exv = put(exv.data(), exv.size() * 4);
     b.off_bnum = put(bnum.data(), bnum.size() * 8);
@@ -587,7 +593,8 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
   if (T == 0) return DAMOE_OK;
   if (T < 0 || T > c->max_T) return fail(c, DAMOE_ERR_INVALID_ARG, "T=%d outside [0, %d]", T, c->max_T);
   if (!x || !w13 || !w2 || !topk_ids || !topk_weights || !out) return fail(c, DAMOE_ERR_INVALID_ARG, "null pointer");
-  if (variant >= c->num_variants() || variant < DAMOE_VARIANT_STATIC) return fail(c, DAMOE_ERR_INVALID_ARG, "variant %d", variant);
+  if (variant < DAMOE_VARIANT_STATIC || (variant >= 0 && !c->variant_ok(variant)))
+    return fail(c, DAMOE_ERR_INVALID_ARG, "variant %d is not available on this context", variant);
   const bool fp8 = c->dtype != DAMOE_BF16;
   if (fp8 && (!c->x_scale || !c->w13_scale || !c->w2_scale))
     return fail(c, DAMOE_ERR_INVALID_ARG, "FP8 context: call damoe_set_fp8_scales first");
@@ -632,10 +639,11 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
     DAMOE_MARK(3);
     DAMOE_CUDA(c, enqueue_gemm(c, pack, 1, known, false, st));
   } else if (c->dispatch == DAMOE_DISPATCH_PREDICATED) {
-    const int nv = c->num_variants();
-    for (int v = 0; v < nv; ++v) DAMOE_CUDA(c, enqueue_gemm(c, pack, 0, v, true, st));
+    for (int v = 0; v < kNumVariants; ++v)
+      if (c->variant_ok(v)) DAMOE_CUDA(c, enqueue_gemm(c, pack, 0, v, true, st));
     DAMOE_MARK(3);
-    for (int v = 0; v < nv; ++v) DAMOE_CUDA(c, enqueue_gemm(c, pack, 1, v, true, st));
+    for (int v = 0; v < kNumVariants; ++v)
+      if (c->variant_ok(v)) DAMOE_CUDA(c, enqueue_gemm(c, pack, 1, v, true, st));
   } else if (fp8) {
     DAMOE_CUDA(c, launch_gemm8(0, -1, false, pack.m13, pack.g13, c->sm_count, st));
     DAMOE_MARK(3);

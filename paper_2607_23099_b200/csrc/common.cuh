@@ -54,14 +54,16 @@ struct VariantDesc {
   int stages13;   // pipeline depth of the gate/up GEMM
   int stages2;    // pipeline depth of the down GEMM
 };
-constexpr int kNumVariants = 7;
-constexpr int kNumVariants1Cta = 5;  // ids 0..4: one CTA per tile; ids 5..6: CTA pairs (cta_group::2, M = 256)
+constexpr int kNumVariants = 8;
+// ids 0..4: one CTA per tile, M = 128 MMAs; ids 5..6: CTA pairs (cta_group::2, M = 256);
+// id 7: the narrowest tile, N = 8, which bf16 MMAs only offer with M = 64 (two per 128-row weight tile)
 __host__ __device__ constexpr VariantDesc variant_desc(int v) {
   constexpr VariantDesc t[kNumVariants] = {
       {16, 128, 1, 6, 10}, {32, 128, 1, 5, 10}, {64, 128, 1, 5, 8}, {128, 128, 1, 4, 6}, {256, 128, 1, 3, 4},
-      {128, 256, 2, 5, 8}, {256, 256, 2, 4, 6}};
+      {128, 256, 2, 5, 8}, {256, 256, 2, 4, 6}, {8, 64, 1, 6, 10}};
   return t[v];
 }
+__host__ __device__ constexpr bool variant_is_pair(int v) { return variant_desc(v).cta_group == 2; }
 
 // What the selector kernel needs to know about the tuning table's bucket for this call.
 struct SelectorArgs {
@@ -127,6 +129,7 @@ struct GemmArgs {
   __nv_bfloat16* h;             // gate/up GEMM output [max_P, I]
   float* y;                     // down GEMM output [max_P, H]
   int E, H, I;
+  int even_split;               // split an expert's tokens evenly over its tiles (else N_v, N_v, ..., rest)
 };
 // variant >= 0: launch that variant's kernel; predicated: it exits unless *variant_id == variant.
 // variant == -1: one kernel that branches on *variant_id.
@@ -154,6 +157,7 @@ struct GemmArgs8 {
   float* hs_T;            // gate/up output scales [I/128, max_P]
   float* y;               // down GEMM output [max_P, H]
   int E, H, I, max_P;
+  int even_split;
 };
 cudaError_t launch_gemm8(int kind, int variant, bool predicated, const GemmMaps& maps, const GemmArgs8& args,
                          int sm_count, cudaStream_t stream);

@@ -55,6 +55,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     case 2: gemm_body<KIND, VCfg<KIND, 2>::kBN, VCfg<KIND, 2>::kStages>(&maps.w, &maps.act[2], a, 2, smem_raw); break;
     case 3: gemm_body<KIND, VCfg<KIND, 3>::kBN, VCfg<KIND, 3>::kStages>(&maps.w, &maps.act[3], a, 3, smem_raw); break;
     case 4: gemm_body<KIND, VCfg<KIND, 4>::kBN, VCfg<KIND, 4>::kStages>(&maps.w, &maps.act[4], a, 4, smem_raw); break;
+    case 7: gemm_body<KIND, VCfg<KIND, 7>::kBN, VCfg<KIND, 7>::kStages>(&maps.w, &maps.act[7], a, 7, smem_raw); break;
     default: break;
   }
 }
@@ -66,6 +67,7 @@ constexpr int max_smem_bytes() {
   m = VCfg<KIND, 2>::C::kSmemBytes > m ? VCfg<KIND, 2>::C::kSmemBytes : m;
   m = VCfg<KIND, 3>::C::kSmemBytes > m ? VCfg<KIND, 3>::C::kSmemBytes : m;
   m = VCfg<KIND, 4>::C::kSmemBytes > m ? VCfg<KIND, 4>::C::kSmemBytes : m;
+  m = VCfg<KIND, 7>::C::kSmemBytes > m ? VCfg<KIND, 7>::C::kSmemBytes : m;
   return m;
 }
 
@@ -92,6 +94,7 @@ cudaError_t launch_kind(int variant, bool predicated, const GemmMaps& maps, cons
     case 2: return launch_fixed<KIND, 2>(maps, args, predicated, grid, stream);
     case 3: return launch_fixed<KIND, 3>(maps, args, predicated, grid, stream);
     case 4: return launch_fixed<KIND, 4>(maps, args, predicated, grid, stream);
+    case 7: return launch_fixed<KIND, 7>(maps, args, predicated, grid, stream);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -102,8 +105,8 @@ cudaError_t gemm_configure() {
   cudaError_t e;
 #define DAMOE_CFG(K, V) \
   if ((e = configure_fixed<K, V>()) != cudaSuccess) return e;
-  DAMOE_CFG(0, 0) DAMOE_CFG(0, 1) DAMOE_CFG(0, 2) DAMOE_CFG(0, 3) DAMOE_CFG(0, 4)
-  DAMOE_CFG(1, 0) DAMOE_CFG(1, 1) DAMOE_CFG(1, 2) DAMOE_CFG(1, 3) DAMOE_CFG(1, 4)
+  DAMOE_CFG(0, 0) DAMOE_CFG(0, 1) DAMOE_CFG(0, 2) DAMOE_CFG(0, 3) DAMOE_CFG(0, 4) DAMOE_CFG(0, 7)
+  DAMOE_CFG(1, 0) DAMOE_CFG(1, 1) DAMOE_CFG(1, 2) DAMOE_CFG(1, 3) DAMOE_CFG(1, 4) DAMOE_CFG(1, 7)
 #undef DAMOE_CFG
   if ((e = cudaFuncSetAttribute(gemm_branch_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 max_smem_bytes<0>())) != cudaSuccess) return e;

@@ -33,6 +33,7 @@ template <int KIND, int BN, int STAGES>
 __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUtensorMap* tmap_act, const GemmArgs& a,
                                           int variant, uint8_t* smem_raw) {
   using C = Cfg<KIND, BN, STAGES>;
+  constexpr bool kHalfM = (BN == 8);
   const int K = (KIND == 0) ? a.H : a.I;
   const int MROWS = (KIND == 0) ? 2 * a.I : a.H;  // weight rows per expert in the [E*rows, K] view
   const int MT = ((KIND == 0) ? a.I : a.H) / kTileM;
@@ -91,7 +92,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
       int it = 0;
       bool ok = true;
       for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
-        const Item item = decode_item(w, s_pref, s_off, E, MT, BN);
+        const Item item = decode_item(w, s_pref, s_off, E, MT, BN, a.even_split);
         const int row_a = item.e * MROWS + item.m_tile * kTileM;
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const int s = it % STAGES;
@@ -122,9 +123,11 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
       for (int w = blockIdx.x; ok && w < total; w += gridDim.x, ++tile_i) {
         // A ragged last token tile issues narrower MMAs: N is a field of the instruction
         // descriptor, so only ceil16(valid) token columns cost tensor time.
-        const Item item = decode_item(w, s_pref, s_off, E, MT, BN);
+        const Item item = decode_item(w, s_pref, s_off, E, MT, BN, a.even_split);
         const int n_eff = (item.valid + 15) & ~15;
-        const uint32_t idesc = umma_idesc_bf16(kTileM, n_eff < BN ? n_eff : BN);
+        // N = 8 exists only with M = 64: the 128-row weight tile is then two MMAs, whose
+        // accumulator rows land in the lower and the upper 16 lanes of each TMEM lane quadrant
+        const uint32_t idesc = kHalfM ? umma_idesc_bf16(64, 8) : umma_idesc_bf16(kTileM, n_eff < BN ? n_eff : BN);
         const int buf = tile_i % C::kNumAcc;
         const uint32_t aph = (tile_i / C::kNumAcc) & 1;
         if (!mbar_wait(bar_tempty + 8u * buf, aph ^ 1u, s_abort)) break;
@@ -147,6 +150,10 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
             const uint32_t acc = (kb | k) ? 1u : 0u;
             umma_bf16(d0, da0 + 2u * k, db + 2u * k, idesc, acc);  // +32 bytes per K=16 step
             if (KIND == 0) umma_bf16(d0 + BN, da1 + 2u * k, db + 2u * k, idesc, acc);
+            if (kHalfM) {  // rows 64..127 of the weight tile: +64 rows * 128 B in shared memory, +16 TMEM lanes
+              umma_bf16(d0 + (16u << 16), da0 + 512u + 2u * k, db + 2u * k, idesc, acc);
+              if (KIND == 0) umma_bf16(d0 + BN + (16u << 16), da1 + 512u + 2u * k, db + 2u * k, idesc, acc);
+            }
           }
           umma_commit(bar_empty + 8u * s);  // stage is free once these MMAs have read it
         }
@@ -158,31 +165,40 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
     const uint32_t lane_base = (warp & 3) * 32;  // the TMEM lane quadrant this warp may read
     int tile_i = 0;
     for (int w = blockIdx.x; w < total; w += gridDim.x, ++tile_i) {
-      const Item item = decode_item(w, s_pref, s_off, E, MT, BN);
+      const Item item = decode_item(w, s_pref, s_off, E, MT, BN, a.even_split);
       const int buf = tile_i % C::kNumAcc;
       const uint32_t aph = (tile_i / C::kNumAcc) & 1;
       if (!mbar_wait(bar_tfull + 8u * buf, aph, s_abort)) break;
       tc_fence_after();
-      const int ch = item.m_tile * kTileM + lane_base + lane;
+      // weight row held by this TMEM lane: lane m for M = 128; for the two M = 64 MMAs lanes
+      // 0..15 of quadrant q hold rows 16q.., lanes 16..31 rows 64 + 16q..
+      const int row = kHalfM ? ((lane < 16 ? 0 : 48) + 16 * static_cast<int>(warp & 3) + lane)
+                             : static_cast<int>(lane_base) + lane;
+      const int ch = item.m_tile * kTileM + row;
       const uint32_t t0 = tmem_base + (lane_base << 16) + buf * C::kAccCols;
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 16) {
         if (c0 >= item.valid) break;
         uint32_t g[16], u[16];
-        tmem_ld_x16(t0 + c0, g);
-        if (KIND == 0) tmem_ld_x16(t0 + BN + c0, u);
+        if constexpr (kHalfM) {
+          tmem_ld_x8(t0 + c0, *reinterpret_cast<uint32_t(*)[8]>(&g[0]));
+          if (KIND == 0) tmem_ld_x8(t0 + BN + c0, *reinterpret_cast<uint32_t(*)[8]>(&u[0]));
+        } else {
+          tmem_ld_x16(t0 + c0, g);
+          if (KIND == 0) tmem_ld_x16(t0 + BN + c0, u);
+        }
         tmem_ld_wait();
         if (KIND == 0) {
           __nv_bfloat16* dst = a.h + static_cast<size_t>(item.q0 + c0) * a.I + ch;
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
+          for (int j = 0; j < (kHalfM ? 8 : 16); ++j)
             if (c0 + j < item.valid)
               dst[static_cast<size_t>(j) * a.I] = __float2bfloat16_rn(silu_mul(__uint_as_float(g[j]), __uint_as_float(u[j])));
         } else {
           float* dst = a.y + static_cast<size_t>(item.q0 + c0) * a.H + ch;
           const float* wq = a.w_sorted + item.q0 + c0;
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
+          for (int j = 0; j < (kHalfM ? 8 : 16); ++j)
             if (c0 + j < item.valid) dst[static_cast<size_t>(j) * a.H] = __ldg(wq + j) * __uint_as_float(g[j]);
         }
       }

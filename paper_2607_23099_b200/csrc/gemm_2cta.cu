@@ -160,7 +160,7 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
       int it = 0;
       bool ok = true;
       for (int w = cluster_id; ok && w < total; w += num_clusters) {
-        const Item item = decode_item(w, s_pref, s_off, E, MT2, BN);   // item.m_tile = pair index
+        const Item item = decode_item(w, s_pref, s_off, E, MT2, BN, a.even_split);   // item.m_tile = pair index
         const int n_eff = (item.valid + 15) & ~15;
         const int n_use = n_eff < BN ? n_eff : BN;
         const int row_a = item.e * MROWS + (2 * item.m_tile + static_cast<int>(rank)) * kTileM;
@@ -188,7 +188,7 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
       int it = 0, tile_i = 0;
       bool ok = true;
       for (int w = cluster_id; ok && w < total; w += num_clusters, ++tile_i) {
-        const Item item = decode_item(w, s_pref, s_off, E, MT2, BN);
+        const Item item = decode_item(w, s_pref, s_off, E, MT2, BN, a.even_split);
         const int n_eff = (item.valid + 15) & ~15;
         const uint32_t idesc = umma_idesc_bf16(2 * kTileM, n_eff < BN ? n_eff : BN);
         const int buf = tile_i % C::kNumAcc;
@@ -224,7 +224,7 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
     const uint32_t lane_base = (warp & 3) * 32;
     int tile_i = 0;
     for (int w = cluster_id; w < total; w += num_clusters, ++tile_i) {
-      const Item item = decode_item(w, s_pref, s_off, E, MT2, BN);
+      const Item item = decode_item(w, s_pref, s_off, E, MT2, BN, a.even_split);
       const int buf = tile_i % C::kNumAcc;
       const uint32_t aph = (tile_i / C::kNumAcc) & 1;
       if (!mbar_wait(bar_tfull + 8u * buf, aph, s_abort)) break;
@@ -310,6 +310,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
     case 4: gemm_body<KIND, VCfg<KIND, 4>::kBN, VCfg<KIND, 4>::kStages>(&maps.w, &maps.act[4], a, 4, smem_raw); break;
     case 5: gemm2_body<KIND, VCfg2<KIND, 5>::kBN, VCfg2<KIND, 5>::kStages>(&maps.w, &maps.act[2], a, 5, smem_raw); break;
     case 6: gemm2_body<KIND, VCfg2<KIND, 6>::kBN, VCfg2<KIND, 6>::kStages>(&maps.w, &maps.act[3], a, 6, smem_raw); break;
+    case 7: gemm_body<KIND, VCfg<KIND, 7>::kBN, VCfg<KIND, 7>::kStages>(&maps.w, &maps.act[7], a, 7, smem_raw); break;
     default: break;
   }
 }
@@ -323,6 +324,7 @@ constexpr int max_smem2() {
   m = VCfg<KIND, 2>::C::kSmemBytes > m ? VCfg<KIND, 2>::C::kSmemBytes : m;
   m = VCfg<KIND, 3>::C::kSmemBytes > m ? VCfg<KIND, 3>::C::kSmemBytes : m;
   m = VCfg<KIND, 4>::C::kSmemBytes > m ? VCfg<KIND, 4>::C::kSmemBytes : m;
+  m = VCfg<KIND, 7>::C::kSmemBytes > m ? VCfg<KIND, 7>::C::kSmemBytes : m;
   return m;
 }
 
