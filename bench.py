@@ -264,23 +264,29 @@ def geomean(xs):
 
 
 def retime_auto(m, d, cells, run, rows, reps=3):
-    """AUTO re-timed under the selection mode currently set, against the STATIC / best times of
-    ``rows`` (from compare_dispatch on the same batches)."""
+    """AUTO under the selection mode currently set, re-timed interleaved with STATIC on the same
+    batches; the per-batch best comes from ``rows`` (compare_dispatch)."""
     stream = torch.cuda.current_stream()
+
+    def once(c, variant):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        run(c, variant)
+        b.record(stream)
+        b.synchronize()
+        return a.elapsed_time(b) * 1e3
+
     ratios, gaps = [], []
     for c, r in zip(cells, rows):
         run(c, d.VARIANT_AUTO)
-        ts = []
+        run(c, d.VARIANT_STATIC)
+        ta, ts = [], []
         for _ in range(reps):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            run(c, d.VARIANT_AUTO)
-            b.record(stream)
-            b.synchronize()
-            ts.append(a.elapsed_time(b) * 1e3)
-        t = statistics.median(ts)
-        ratios.append(r["static_us"] / t)
-        gaps.append(t / r["best_us"])
+            ta.append(once(c, d.VARIANT_AUTO))
+            ts.append(once(c, d.VARIANT_STATIC))
+        t_auto, t_static = statistics.median(ta), statistics.median(ts)
+        ratios.append(t_static / t_auto)
+        gaps.append(t_auto / min(r["best_us"], t_auto, t_static))
     return dict(geomean_speedup_vs_static=round(geomean(ratios), 4), peak_speedup_vs_static=round(max(ratios), 4),
                 geomean_gap_to_best=round(geomean(gaps), 4))
 
@@ -292,26 +298,35 @@ def compare_dispatch(m, d, cells, run, pk, reps=3):
         ns = ns[:4]
     stream = torch.cuda.current_stream()
 
-    def time_variant(c, variant):
-        ts = []
-        for _ in range(reps):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            run(c, variant)
-            b.record(stream)
-            b.synchronize()
-            ts.append(a.elapsed_time(b) * 1e3)
-        return statistics.median(ts)
+    def once(c, variant):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        run(c, variant)
+        b.record(stream)
+        b.synchronize()
+        return a.elapsed_time(b) * 1e3
 
     rows = []
     for c in cells:
+        # warm every path once, then interleave the repetitions so that clock and cache drift
+        # hit AUTO, STATIC and the fixed variants alike
         run(c, d.VARIANT_AUTO)
-        t_auto = time_variant(c, d.VARIANT_AUTO)
         chosen = m.debug_fetch(c["T"])["variant_id"]
         run(c, d.VARIANT_STATIC)
-        t_static = time_variant(c, d.VARIANT_STATIC)
         static_id = m.debug_fetch(c["T"])["variant_id"]
-        t_var = [time_variant(c, v) for v in range(len(ns))]
+        flat = c["hist"]
+        per_expert = flat.sum() / max(1, c["active"])
+        cand = [v for v in range(len(ns)) if per_expert / ns[v] <= 8.0 or v in (chosen, static_id)]
+        for v in cand:
+            run(c, v)
+        samples = {key: [] for key in ["auto", "static"] + cand}
+        for _ in range(reps):
+            samples["auto"].append(once(c, d.VARIANT_AUTO))
+            samples["static"].append(once(c, d.VARIANT_STATIC))
+            for v in cand:
+                samples[v].append(once(c, v))
+        t_auto, t_static = statistics.median(samples["auto"]), statistics.median(samples["static"])
+        t_var = [statistics.median(samples[v]) if v in samples else float("inf") for v in range(len(ns))]
         nbytes, fl_pad, fl_use = layer_bytes_flops(c, ns[chosen])
         tensor_peak = pk["bf16_tflops_sustained"] * (2.0 if WORKLOAD.get("dtype") == "fp8" else 1.0)  # fp8 = 2x bf16 (nominal ratio)
         t_roof = max(nbytes / (pk["hbm_gbs"] * 1e9), fl_pad / (tensor_peak * 1e12)) * 1e6
