@@ -177,6 +177,8 @@ def sweep(shape, buckets, alphas, seeds, reps, log_path, weight_seed=12345, devi
     else:
         w13, w2 = W.materialize(device)
     m = d.DAMoE(max(buckets), k, E, H, I, dtype=dtype)
+    if log_path:
+        os.makedirs(os.path.dirname(os.path.abspath(log_path)), exist_ok=True)
     log = open(log_path, "a") if log_path else None
     result = {}
     for T in buckets:

@@ -8,10 +8,12 @@
 // buffer.  Everything else follows the bf16 kernel: swap-AB, persistent CTAs decoding work
 // items from the device-side tile prefix, TMA-fed multistage ring, bounded waits.
 //
-// CTA = 10 warps: warp 0 TMA producer, warp 1 MMA issuer + TMEM allocation, warps 2..9
-// epilogue; epilogue warp pairs (w, w+4) share a TMEM lane quadrant and split the token
-// columns in halves, which keeps the register accumulators at N_v (gate/up) or N_v/2 (down)
-// floats per thread.
+// CTA = 18 warps: warp 0 TMA producer, warp 1 MMA issuer + TMEM allocation, warps 2..17
+// epilogue: four warps per TMEM lane quadrant (two for the narrowest tile), each owning a group of
+// N_v / 4 token columns.  Every K block has to pass through all epilogue warps, so the promotion
+// rate is set by the work of ONE warp per K block; spreading the columns over four groups (and
+// four warps per scheduler to hide the TMEM-load and shuffle latencies) is what keeps it from
+// throttling the MMAs, and it keeps the register accumulators at N_v / 2 floats per thread.
 //
 // KIND 0 (gate/up): a = silu(g) * u, h_b = bf16(a); the 128 channels of the weight tile are
 //   exactly one 1x128 scale group of h, so the group amax is a reduction over the tile's 128
@@ -27,7 +29,7 @@ namespace damoe {
 
 namespace {
 
-constexpr int kThreads8 = 320;
+constexpr int kThreads8 = 576;  // 2 + 16 warps
 constexpr int kABytes8 = kTileM * kBK8;  // 128 rows x 128 one-byte elements
 constexpr int kTailBytes8 = 2 * (kMaxE + 1) * 4 + 512 + 2 * 4 * 128 * 4;  // + amax exchange, double-buffered [2][4 quadrants][BN <= 128]
 
@@ -58,7 +60,8 @@ struct Cfg8 {
   static constexpr int kTmemColsRaw = kNumPartials * kAccCols;
   static constexpr int kTmemCols = kTmemColsRaw <= 32 ? 32 : kTmemColsRaw <= 64 ? 64 : kTmemColsRaw <= 128 ? 128
                                    : kTmemColsRaw <= 256 ? 256 : 512;
-  static constexpr int kCW = BN / 2;              // token columns per epilogue warp
+  static constexpr int kGroups = (BN >= 32) ? 4 : 2;   // column groups: epilogue warps per TMEM lane quadrant
+  static constexpr int kCW = BN / kGroups;          // token columns per epilogue warp
   static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + kTailBytes8;
   static_assert(kTmemColsRaw <= 512, "partials do not fit TMEM");
   static_assert(kStageBytes % 1024 == 0, "operand tiles must stay 1024-byte aligned for the 128B swizzle");
@@ -105,8 +108,9 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
   const uint32_t bar_empty = bar_full + 8u * STAGES;
   const uint32_t bar_pfull = bar_empty + 8u * STAGES;
   const uint32_t bar_pempty = bar_pfull + 32u;
-  const uint32_t bar_xchg = bar_pempty + 32u;  // one per column half: the 4 warps sharing it exchange amax
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 10);
+  const uint32_t bar_xchg = bar_pempty + 32u;  // one per column group: the 4 warps sharing it exchange amax
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 12);
+  constexpr int G = C::kGroups;
   constexpr int NP = C::kNumPartials;
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   float* s_amax = reinterpret_cast<float*>(s_tmem + 2);  // [2 buffers][4 quadrants][BN]
@@ -127,9 +131,9 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
     }
     for (int b = 0; b < 4; ++b) {
       mbar_init(bar_pfull + 8u * b, 1);
-      mbar_init(bar_pempty + 8u * b, 8);
+      mbar_init(bar_pempty + 8u * b, 4 * G);
+      mbar_init(bar_xchg + 8u * b, 4);
     }
-    for (int b = 0; b < 2; ++b) mbar_init(bar_xchg + 8u * b, 4);
     *s_abort = 0;
     fence_mbar_init();
     fence_proxy_async_smem();
@@ -211,15 +215,15 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
     }
   } else {
     // ---------------- epilogue warps: scale promotion, then the fused output ----------------
-    const int ew = warp - 2;                        // 0..7
+    const int ew = warp - 2;                        // 0..15
     const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
-    const int half = ew >> 2;                       // which half of the token columns
+    const int half = ew >> 2;                       // which group of token columns (named half for two groups)
     const uint32_t lane_base = quad * 32;
     const int col0 = half * CW;
     const int wblocks_k = K / 128;
     const float* wsc = a.w_scale;
     int it = 0, item_i = 0;
-    for (int w = blockIdx.x; w < total; w += gridDim.x, ++item_i) {
+    for (int w = blockIdx.x; half < G && w < total; w += gridDim.x, ++item_i) {
       const Item item = decode_item(w, s_pref, s_off, E, MT, BN, a.even_split);
       const int ch = item.m_tile * kTileM + lane_base + lane;
       // weight-scale rows of this item: [expert, row block, K block]
