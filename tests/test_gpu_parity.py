@@ -262,6 +262,38 @@ def test_graph_switch_dispatch(d):
     m.close()
 
 
+def test_capture_in_a_cuda_graph(d):
+    # the layer call only enqueues kernels: captured once, replayed on new routing written into the same buffers
+    E, k, H, I, T = 8, 2, 1024, 512, 48
+    W = di.MoEWeights(4, E, H, I)
+    w13, w2 = W.materialize("cuda")
+    m = d.DAMoE(64, k, E, H, I)
+    ids_d = torch.zeros(T, k, dtype=torch.int32, device="cuda")
+    w_d = torch.zeros(T, k, dtype=torch.float32, device="cuda")
+    x_d = torch.zeros(T, H, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(T, H, dtype=torch.bfloat16, device="cuda")
+    first = Case(20, T, E, k, H, I, 1.0)
+    ids_d.copy_(torch.from_numpy(first.ids)); w_d.copy_(torch.from_numpy(first.w)); x_d.copy_(first.x("cuda"))
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        m.fused_moe(x_d, w13, w2, ids_d, w_d, d.VARIANT_AUTO, out=out, stream=side)    # warm-up outside the capture
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        m.fused_moe(x_d, w13, w2, ids_d, w_d, d.VARIANT_AUTO, out=out, stream=side)
+    for seed, alpha in [(21, 0.1), (22, 10.0)]:
+        case = Case(seed, T, E, k, H, I, alpha)
+        case.weights = W
+        ids_d.copy_(torch.from_numpy(case.ids)); w_d.copy_(torch.from_numpy(case.w)); x_d.copy_(case.x("cuda"))
+        graph.replay()
+        torch.cuda.synchronize()
+        meta = m.debug_fetch(T)
+        assert meta["status"] == 0
+        _check_route(meta, case, d.tile_ns())
+        _check_layer(out, case)
+    m.close()
+
+
 def test_host_buffer_entry_point(d):
     case = config0(seed=6, T=32)
     t = _device_case(case)
