@@ -58,6 +58,15 @@ TRACE_WORKLOAD = dict(name="kimi_k2_trace_500", E=384, k=8, H=7168, I=2048, T=40
 # scales, bf16 output; T in {16, 256, 4096} x alpha in {0.1, 1, 10}.
 FP8_WORKLOAD = dict(name="deepseek_v3_fp8_grid", E=256, k=8, H=7168, I=2048, T=4096, dtype="fp8",
                     grid=[(T, a) for T in (16, 256, 4096) for a in (0.1, 1.0, 10.0)], weight_seed=12345)
+# Kernel-variant landscape on the headline shape: T in {1, 4, 16, 64, 256, 1024, 4096, 8192} x
+# alpha in {0.05, 0.2, 1, 10}, one batch per cell; every cell reports its roofline fraction.
+GRID_WORKLOAD = dict(name="deepseek_v3_landscape_grid", E=256, k=8, H=7168, I=2048, T=8192,
+                     grid=[(T, a) for T in (1, 4, 16, 64, 256, 1024, 4096, 8192) for a in (0.05, 0.2, 1.0, 10.0)],
+                     weight_seed=12345)
+# Prefill-sized batches on the headline shape (about 256 tokens per expert): the tensor-bound,
+# power-capped end of the landscape, timed alone so that the sampled clocks are those of this regime.
+LARGE_T_WORKLOAD = dict(name="deepseek_v3_prefill_T8192", E=256, k=8, H=7168, I=2048, T=8192,
+                        alphas=[1.0, 10.0], seeds=[0, 1], weight_seed=12345)
 # One expert-parallel shard (EP = 4) of the DeepSeek-V3 layer on one GPU: 64 local experts, routing
 # drawn over all 256 experts and masked to the shard; 200 batches, T log-uniform in [1, 2048].
 EP4_WORKLOAD = dict(name="deepseek_v3_ep4_shard_trace_200", E=64, E_global=256, k=8, H=7168, I=2048, T=2048,
@@ -150,18 +159,20 @@ class ClockSampler:
         time.sleep(0.15)
         self.proc.terminate()
         rows = [r for t, r in self.rows if t0 <= t <= t1 + 0.11] or [r for _, r in self.rows]
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         for r in rows:
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
+                pw.append(float(r[2]))
             except (ValueError, IndexError):
                 continue
             for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
-                    reasons=sorted(reasons), samples=len(sm))
+                    reasons=sorted(reasons), samples=len(sm), sm_mhz_min=min(sm) if sm else None,
+                    power_w=statistics.median(pw) if pw else None)
 
 
 def layer_bytes_flops(cell, tile_n):
@@ -512,13 +523,25 @@ def run_ours(args):
     achieved = w13_bytes / (w13_ms * 1e-3) / 1e9
     # the ncu capture is of the bf16 kernel at ~2 tokens per expert; it is only scaled to workloads of that kind
     traffic = None
-    if not fp8 and not is_trace:
+    if not fp8 and not is_trace and "grid" not in w:
         traffic = round(NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 * statistics.mean(c["active"] for c in rec_cells))
-    roofline = dict(bound="hbm", kernel=("gemm8_branch_kernel<0>" if fp8 else "gemm2_branch_kernel<0>") + " (grouped gate/up GEMM + SwiGLU, branching on the device-side variant id)", achieved=round(achieved, 1),
-                    peak=pk["hbm_gbs"], unit="GB/s", frac=round(achieved / pk["hbm_gbs"], 4), traffic=traffic,
-                    algorithmic_bytes=round(w13_bytes), peak_source=pk["source"], launch_ms=round(w13_ms, 4),
-                    launches_timed=n_rec,
-                    stage_share={k: round(stage[k] / max(1e-9, sum(stage[s] for s in m.STAGES)), 4) for k in m.STAGES})
+    kernel_name = ("gemm8_branch_kernel<0>" if fp8 else "gemm2_branch_kernel<0>") + \
+        " (grouped gate/up GEMM + SwiGLU, branching on the device-side variant id)"
+    share = {k: round(stage[k] / max(1e-9, sum(stage[s] for s in m.STAGES)), 4) for k in m.STAGES}
+    # the gate/up GEMM's own two bounds: its bytes over HBM, its useful flops over the tensor peak
+    w13_flops = statistics.mean(float(c["hist"].sum()) * 4 * w["H"] * w["I"] for c in rec_cells)
+    tensor_peak = pk["bf16_tflops_sustained"] * (2.0 if fp8 else 1.0)
+    if w13_flops / (tensor_peak * 1e12) > w13_bytes / (pk["hbm_gbs"] * 1e9):
+        tf = w13_flops / (w13_ms * 1e-3) / 1e12
+        roofline = dict(bound="tensor", kernel=kernel_name, achieved=round(tf, 1), peak=tensor_peak, unit="TFLOP/s",
+                        frac=round(tf / tensor_peak, 4), traffic=None, algorithmic_flops=round(w13_flops),
+                        peak_source=pk["source"] + " (sustained cuBLAS bf16" + (", x2 nominal ratio for fp8)" if fp8 else ")"),
+                        launch_ms=round(w13_ms, 4), launches_timed=n_rec, stage_share=share)
+    else:
+        roofline = dict(bound="hbm", kernel=kernel_name, achieved=round(achieved, 1),
+                        peak=pk["hbm_gbs"], unit="GB/s", frac=round(achieved / pk["hbm_gbs"], 4), traffic=traffic,
+                        algorithmic_bytes=round(w13_bytes), peak_source=pk["source"], launch_ms=round(w13_ms, 4),
+                        launches_timed=n_rec, stage_share=share)
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -539,7 +562,7 @@ def run_ours(args):
     if "alphas" in w:
         config.update(alphas=w["alphas"], seeds_per_alpha=len(w["seeds"]))
     if "grid" in w:
-        config.update(T="{16, 256, 4096}", alphas=[0.1, 1.0, 10.0])
+        config.update(T=sorted({T for T, _ in w["grid"]}), alphas=sorted({a for _, a in w["grid"]}))
     if fp8:
         config.update(e2e_note="host-buffer entry point is bf16 only; e2e repeats the device-timed call")
     line = dict(metric="fused_moe_layer_us", value=round(us_per_layer, 2), unit="us", n_gpus=world, steps=steps,
@@ -560,7 +583,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="headline", choices=["headline", "small", "small_dense", "mid_dense", "small_dense_fp8", "kimi_trace", "fp8_grid", "ep4_trace"],
+    ap.add_argument("--workload", default="headline", choices=["headline", "small", "small_dense", "mid_dense", "small_dense_fp8", "kimi_trace", "fp8_grid", "ep4_trace", "bf16_grid", "large_T"],
                     help="'small' is the reduced case used for ncu captures; 'kimi_trace' the 500-batch serving-trace stand-in")
     ap.add_argument("--no-table", action="store_true", help="ignore the committed tuning table")
     ap.add_argument("--table", default=None, help="tuning table file to load instead of the committed one")
@@ -570,7 +593,7 @@ def main():
         WORKLOAD.clear()
         WORKLOAD.update(dict(small=SMALL_WORKLOAD, small_dense=SMALL_DENSE_WORKLOAD, mid_dense=MID_DENSE_WORKLOAD, small_dense_fp8=SMALL_DENSE_FP8_WORKLOAD,
                              kimi_trace=TRACE_WORKLOAD, fp8_grid=FP8_WORKLOAD,
-                             ep4_trace=EP4_WORKLOAD)[args.workload])
+                             ep4_trace=EP4_WORKLOAD, bf16_grid=GRID_WORKLOAD, large_T=LARGE_T_WORKLOAD)[args.workload])
     if args.impl == "reference":
         run_reference(args)
     else:
