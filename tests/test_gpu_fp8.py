@@ -104,8 +104,9 @@ def test_fp8_config4_shape_sampled_tokens(d):
     E, k, H, I = 256, 8, 7168, 2048
     W = di.MoEWeights(12345, E, H, I)
     wq = W.materialize_fp8("cuda:0")
-    m = d.DAMoE(256, k, E, H, I, dtype=d.FP8_E4M3_BLOCK128)
-    for T, alpha, seed, variant in [(16, 0.1, 0, d.VARIANT_AUTO), (256, 10.0, 1, 1), (256, 1.0, 2, 3)]:
+    m = d.DAMoE(4096, k, E, H, I, dtype=d.FP8_E4M3_BLOCK128)
+    for T, alpha, seed, variant in [(16, 0.1, 0, d.VARIANT_AUTO), (256, 10.0, 1, 1), (256, 1.0, 2, 3),
+                                    (4096, 1.0, 3, d.VARIANT_AUTO), (4096, 0.1, 4, 3)]:
         case = Fp8Case(seed, T, E, k, H, I, alpha, weights=W)
         out, meta = _run(d, m, case, wq, variant)
         assert meta["status"] == 0

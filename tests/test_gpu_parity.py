@@ -324,6 +324,49 @@ def test_config1_shape_sampled_tokens(d):
     m.close()
 
 
+def _table_bytes(E, k, H, I, dtype="bf16"):
+    import os
+    import paper_2607_23099_b200 as pkg
+    path = os.path.join(os.path.dirname(pkg.__file__), "tables", f"e{E}_k{k}_h{H}_i{I}_{dtype}.damoetb")
+    return open(path, "rb").read()
+
+
+def _sampled_full_size(d, E, k, H, I, max_T, cells):
+    # The launch configuration the benchmark times: shipped tuning table, AUTO, in-kernel branch.
+    W = di.MoEWeights(12345, E, H, I)
+    w13, w2 = W.materialize("cuda")
+    m = d.DAMoE(max_T, k, E, H, I)
+    m.load_tuning_table(_table_bytes(E, k, H, I))
+    ns = d.tile_ns()
+    for T, alpha, seed in cells:
+        case = Case(seed, T, E, k, H, I, alpha)
+        case.weights = W
+        out = m.fused_moe(case.x("cuda"), w13, w2, torch.from_numpy(case.ids).cuda(), torch.from_numpy(case.w).cuda(),
+                          d.VARIANT_AUTO)
+        meta = m.debug_fetch(T)
+        assert meta["status"] == 0
+        _check_route(meta, case, ns)
+        assert 0 <= meta["variant_id"] < len(ns)
+        tokens = sorted(int(v) for v in np.random.default_rng(seed).choice(T, size=min(2, T), replace=False))
+        _check_layer(out, case, tokens=tokens)
+        # rows of tokens that were not sampled must be finite too (a missed tile would leave garbage or zeros)
+        got = codecs.bf16_decode(bits16(out))
+        assert np.all(np.isfinite(got))
+        assert np.all(np.abs(got).max(axis=1) > 0)
+    m.close()
+
+
+def test_config2_landscape_large_T_sampled_tokens(d):
+    # The largest cells of the kernel-variant landscape on the DeepSeek-V3 shape: prefill-sized
+    # batches, skewed and near-uniform (CTA-pair variants, several token tiles per expert).
+    _sampled_full_size(d, 256, 8, 7168, 2048, 8192, [(8192, 1.0, 11), (4096, 0.05, 12), (1024, 0.2, 13)])
+
+
+def test_config3_kimi_shape_sampled_tokens(d):
+    # Kimi-K2-shaped layer (E=384): one decode-sized, one ragged mid-sized and the largest batch of the trace.
+    _sampled_full_size(d, 384, 8, 7168, 2048, 4096, [(1, 1.0, 21), (333, 0.3, 22), (4096, 5.0, 23)])
+
+
 def test_dispatch_microbench_runs(d):
     r = d.dispatch_microbench(50)
     assert all(0 < v < 1e4 for v in r.values())
