@@ -34,9 +34,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     gemm_fixed_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_act,
                       const GemmArgs a, const int predicated) {
   extern __shared__ uint8_t smem_raw[];
-  if (predicated) {
-    pdl_launch_dependents();
+  if (predicated) {  // a kernel that is not selected still waits: its completion orders the kernels after it
     pdl_wait();
+    pdl_launch_dependents();
     if (*a.variant_id != V) return;
   }
   gemm_body<KIND, VCfg<KIND, V>::kBN, VCfg<KIND, V>::kStages>(&tmap_w, &tmap_act, a, V, smem_raw);
@@ -46,9 +46,7 @@ template <int KIND>
 __global__ void __launch_bounds__(kGemmThreads, 1)
     gemm_branch_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
   extern __shared__ uint8_t smem_raw[];
-  pdl_launch_dependents();
-  pdl_wait();
-  const int v = *a.variant_id;
+  const int v = *a.variant_id;  // written by the route kernel, at least two kernels upstream (see gemm_body)
   switch (v) {
     case 0: gemm_body<KIND, VCfg<KIND, 0>::kBN, VCfg<KIND, 0>::kStages>(&maps.w, &maps.act[0], a, 0, smem_raw); break;
     case 1: gemm_body<KIND, VCfg<KIND, 1>::kBN, VCfg<KIND, 1>::kStages>(&maps.w, &maps.act[1], a, 1, smem_raw); break;
@@ -56,7 +54,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     case 3: gemm_body<KIND, VCfg<KIND, 3>::kBN, VCfg<KIND, 3>::kStages>(&maps.w, &maps.act[3], a, 3, smem_raw); break;
     case 4: gemm_body<KIND, VCfg<KIND, 4>::kBN, VCfg<KIND, 4>::kStages>(&maps.w, &maps.act[4], a, 4, smem_raw); break;
     case 7: gemm_body<KIND, VCfg<KIND, 7>::kBN, VCfg<KIND, 7>::kStages>(&maps.w, &maps.act[7], a, 7, smem_raw); break;
-    default: break;
+    default:  // no such variant: still order the kernels after this one behind the kernel before it
+      pdl_wait();
+      pdl_launch_dependents();
+      break;
   }
 }
 

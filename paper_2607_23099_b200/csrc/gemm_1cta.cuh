@@ -54,8 +54,11 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-  pdl_launch_dependents();
-  pdl_wait();  // everything below reads what the route / gather / previous GEMM kernels wrote
+  // Programmatic dependent launch: this kernel may start while the kernel before it in the
+  // stream (the gather, or the gate/up GEMM) is still running.  Every kernel of the layer
+  // releases its dependents only AFTER its own wait, so by the time a CTA of this kernel runs,
+  // everything two or more kernels upstream - the routing metadata - is complete and may be
+  // read at once; only the activations (the B operand) need the wait below.
   const int32_t* pref_g = a.ntile_prefix + variant * (E + 1);
   for (int i = tid; i <= E; i += kGemmThreads) {
     s_pref[i] = pref_g[i];
@@ -85,27 +88,49 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
   const int total = s_pref[E] * MT;
+  if (tid != 0) {  // thread 0 (the producer) waits after it has issued the first weight loads
+    pdl_wait();
+    pdl_launch_dependents();
+  }
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       int it = 0;
       bool ok = true;
+      // The weights of the first item start streaming before the upstream kernel has finished.
+      int n_pre = 0;
+      if (static_cast<int>(blockIdx.x) < total) {
+        const Item item = decode_item(blockIdx.x, s_pref, s_off, E, MT, BN, a.even_split);
+        const int row_a = item.e * MROWS + item.m_tile * kTileM;
+        n_pre = KB < STAGES ? KB : STAGES;
+        for (int kb = 0; kb < n_pre; ++kb) {
+          const uint32_t full = bar_full + 8u * kb;
+          const uint32_t sa = tiles_base + kb * C::kStageBytes;
+          mbar_arrive_expect_tx(full, C::kStageBytes);  // the activations' bytes follow after the wait
+          tma_load_2d(sa, tmap_w, full, kb * kBK, row_a);
+          if (KIND == 0) tma_load_2d(sa + kABytes, tmap_w, full, kb * kBK, row_a + a.I);
+        }
+      }
+      pdl_wait();
+      pdl_launch_dependents();
       for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
         const Item item = decode_item(w, s_pref, s_off, E, MT, BN, a.even_split);
         const int row_a = item.e * MROWS + item.m_tile * kTileM;
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
-          if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, s_abort)) {
-            ok = false;
-            break;
-          }
           const uint32_t full = bar_full + 8u * s;
           const uint32_t sa = tiles_base + s * C::kStageBytes;
-          mbar_arrive_expect_tx(full, C::kStageBytes);
-          tma_load_2d(sa, tmap_w, full, kb * kBK, row_a);
-          if (KIND == 0) tma_load_2d(sa + kABytes, tmap_w, full, kb * kBK, row_a + a.I);
+          if (it >= n_pre) {
+            const uint32_t ph = (it / STAGES) & 1;
+            if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, s_abort)) {
+              ok = false;
+              break;
+            }
+            mbar_arrive_expect_tx(full, C::kStageBytes);
+            tma_load_2d(sa, tmap_w, full, kb * kBK, row_a);
+            if (KIND == 0) tma_load_2d(sa + kABytes, tmap_w, full, kb * kBK, row_a + a.I);
+          }
           tma_load_2d(sa + C::kATiles * kABytes, tmap_act, full, kb * kBK, item.q0);
         }
       }

@@ -121,8 +121,8 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-  pdl_launch_dependents();
-  pdl_wait();
+  // As in the 1-CTA body: the routing metadata is complete when this kernel starts, the first
+  // item's weights are requested before the wait, and dependents are released after it.
   const int32_t* pref_g = a.ntile_prefix + variant * (E + 1);
   for (int i = tid; i <= E; i += kThreads2) {
     s_pref[i] = pref_g[i];
@@ -153,12 +153,31 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
   const int total = s_pref[E] * MT2;
+  if (tid != 0) {  // thread 0 (the producer) waits after it has issued the first weight loads
+    pdl_wait();
+    pdl_launch_dependents();
+  }
 
   if (warp == 0) {
     // ---------------- TMA producer (both CTAs) ----------------
     if (lane == 0) {
       int it = 0;
       bool ok = true;
+      int n_pre = 0;
+      if (cluster_id < total) {  // the first item's weights, before the upstream kernel has finished
+        const Item item = decode_item(cluster_id, s_pref, s_off, E, MT2, BN, a.even_split);
+        const int row_a = item.e * MROWS + (2 * item.m_tile + static_cast<int>(rank)) * kTileM;
+        n_pre = KB < STAGES ? KB : STAGES;
+        for (int kb = 0; kb < n_pre; ++kb) {
+          const uint32_t full_leader = map_to_cta(bar_full + 8u * kb, 0);
+          const uint32_t sa = tiles_base + kb * C::kStageBytes;
+          if (rank == 0) mbar_arrive_expect_tx(bar_full + 8u * kb, 2u * C::kStageBytes);  // both CTAs' bytes, activations included
+          tma_load_2d_pair(sa, tmap_w, full_leader, kb * kBK, row_a);
+          if (KIND == 0) tma_load_2d_pair(sa + kABytes2, tmap_w, full_leader, kb * kBK, row_a + a.I);
+        }
+      }
+      pdl_wait();
+      pdl_launch_dependents();
       for (int w = cluster_id; ok && w < total; w += num_clusters) {
         const Item item = decode_item(w, s_pref, s_off, E, MT2, BN, a.even_split);   // item.m_tile = pair index
         const int n_eff = (item.valid + 15) & ~15;
@@ -167,16 +186,18 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
         const int row_b = item.q0 + static_cast<int>(rank) * (n_use >> 1);  // this CTA's half of the token columns
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
-          if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, s_abort)) {
-            ok = false;
-            break;
-          }
           const uint32_t full_leader = map_to_cta(bar_full + 8u * s, 0);
           const uint32_t sa = tiles_base + s * C::kStageBytes;
-          if (rank == 0) mbar_arrive_expect_tx(bar_full + 8u * s, 2u * C::kStageBytes);  // both CTAs' bytes
-          tma_load_2d_pair(sa, tmap_w, full_leader, kb * kBK, row_a);
-          if (KIND == 0) tma_load_2d_pair(sa + kABytes2, tmap_w, full_leader, kb * kBK, row_a + a.I);
+          if (it >= n_pre) {
+            const uint32_t ph = (it / STAGES) & 1;
+            if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, s_abort)) {
+              ok = false;
+              break;
+            }
+            if (rank == 0) mbar_arrive_expect_tx(bar_full + 8u * s, 2u * C::kStageBytes);  // both CTAs' bytes
+            tma_load_2d_pair(sa, tmap_w, full_leader, kb * kBK, row_a);
+            if (KIND == 0) tma_load_2d_pair(sa + kABytes2, tmap_w, full_leader, kb * kBK, row_a + a.I);
+          }
           tma_load_2d_pair(sa + C::kATiles * kABytes2, tmap_act, full_leader, kb * kBK, row_b);
         }
       }
@@ -285,9 +306,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
     gemm2_fixed_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_act,
                        const GemmArgs a, const int predicated) {
   extern __shared__ uint8_t smem_raw[];
-  if (predicated) {
-    pdl_launch_dependents();
+  if (predicated) {  // a kernel that is not selected still waits: its completion orders the kernels after it
     pdl_wait();
+    pdl_launch_dependents();
     if (*a.variant_id != V) return;
   }
   gemm2_body<KIND, VCfg2<KIND, V>::kBN, VCfg2<KIND, V>::kStages>(&tmap_w, &tmap_act, a, V, smem_raw);
@@ -299,9 +320,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
   extern __shared__ uint8_t smem_raw[];
   // One launch covers the whole family: the 1-CTA variants simply ignore that they were
   // launched as clusters of two, the CTA-pair variants use it.
-  pdl_launch_dependents();
-  pdl_wait();
-  const int v = *a.variant_id;
+  const int v = *a.variant_id;  // written by the route kernel, at least two kernels upstream; the bodies wait
   switch (v) {
     case 0: gemm_body<KIND, VCfg<KIND, 0>::kBN, VCfg<KIND, 0>::kStages>(&maps.w, &maps.act[0], a, 0, smem_raw); break;
     case 1: gemm_body<KIND, VCfg<KIND, 1>::kBN, VCfg<KIND, 1>::kStages>(&maps.w, &maps.act[1], a, 1, smem_raw); break;
@@ -311,7 +330,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
     case 5: gemm2_body<KIND, VCfg2<KIND, 5>::kBN, VCfg2<KIND, 5>::kStages>(&maps.w, &maps.act[2], a, 5, smem_raw); break;
     case 6: gemm2_body<KIND, VCfg2<KIND, 6>::kBN, VCfg2<KIND, 6>::kStages>(&maps.w, &maps.act[3], a, 6, smem_raw); break;
     case 7: gemm_body<KIND, VCfg<KIND, 7>::kBN, VCfg<KIND, 7>::kStages>(&maps.w, &maps.act[7], a, 7, smem_raw); break;
-    default: break;
+    default:  // no such variant: still order the kernels after this one behind the kernel before it
+      pdl_wait();
+      pdl_launch_dependents();
+      break;
   }
 }
 

@@ -117,8 +117,8 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int32_t* pref_g = a.ntile_prefix + variant * (E + 1);
   for (int i = tid; i <= E; i += kThreads8) {
     s_pref[i] = pref_g[i];
@@ -362,8 +362,8 @@ __global__ void __launch_bounds__(kThreads8, 1)
                        const GemmArgs8 a, const int predicated) {
   extern __shared__ uint8_t smem_raw[];
   if (predicated) {
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();
     if (*a.variant_id != V) return;
   }
   gemm8_body<KIND, VCfg8<KIND, V>::kBN, VCfg8<KIND, V>::kStages>(&tmap_w, &tmap_act, a, V, smem_raw);
@@ -373,8 +373,8 @@ template <int KIND>
 __global__ void __launch_bounds__(kThreads8, 1)
     gemm8_branch_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs8 a) {
   extern __shared__ uint8_t smem_raw[];
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int v = *a.variant_id;
   switch (v) {
     case 0: gemm8_body<KIND, VCfg8<KIND, 0>::kBN, VCfg8<KIND, 0>::kStages>(&maps.w, &maps.act[0], a, 0, smem_raw); break;
@@ -420,8 +420,8 @@ __global__ void __launch_bounds__(256) gather_rows8_kernel(const uint4* __restri
                                                            const int32_t* __restrict__ perm, int k, int row_vec,
                                                            int nblk, int max_P) {
   const int q = blockIdx.x;
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int p = perm[q];
   if (p < 0) return;
   const int t = p / k;

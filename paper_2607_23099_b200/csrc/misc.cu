@@ -11,8 +11,8 @@ namespace {
 __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restrict__ x, uint4* __restrict__ x_perm,
                                                           const int32_t* __restrict__ perm, int k, int row_vec) {
   const int q = blockIdx.x;
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int p = perm[q];
   if (p < 0) return;
   const uint4* src = x + static_cast<size_t>(p / k) * row_vec;
@@ -27,8 +27,8 @@ __global__ void __launch_bounds__(256) unpermute_reduce_kernel(const float4* __r
                                                                uint2* __restrict__ out, int k, int row_vec) {
   const int t = blockIdx.x;
   __shared__ int s_q[kMaxK];
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   if (threadIdx.x < k) s_q[threadIdx.x] = inv[t * k + threadIdx.x];
   __syncthreads();
   for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < row_vec; i += gridDim.y * blockDim.x) {

@@ -25,10 +25,10 @@ __global__ void __launch_bounds__(kPairsPerBlock) route_count_kernel(const int32
                                                                      int32_t* __restrict__ block_hist,
                                                                      uint32_t* __restrict__ status) {
   __shared__ int s_hist[kMaxE];
-  pdl_launch_dependents();
   for (int e = threadIdx.x; e < E; e += blockDim.x) s_hist[e] = 0;
   __syncthreads();
   pdl_wait();
+  pdl_launch_dependents();  // after the wait: a kernel downstream may then read, before its own wait, what the kernel before this one wrote
   const int p = blockIdx.x * kPairsPerBlock + threadIdx.x;
   const int lane = threadIdx.x & 31;
   const int e = (p < P) ? ids[p] : -1;
@@ -141,7 +141,6 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
   __shared__ long long s_score[kMaxExemplars];
   __shared__ int s_active;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  pdl_launch_dependents();
   const bool select = !stats_only && sel.forced < 0;
   const bool ex_staged = select && sel.mode == DAMOE_MODE_EXEMPLAR && sel.n_exemplars * E <= kExPrefetchInts;
   if (select && sel.mode == DAMOE_MODE_EXEMPLAR) {
@@ -156,6 +155,7 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
   }
   __syncthreads();
   pdl_wait();
+  pdl_launch_dependents();  // after the wait: a kernel downstream may then read, before its own wait, what the kernel before this one wrote
 
   if (FUSED) {
     const int e = (tid < P) ? ids[tid] : -1;
@@ -378,10 +378,10 @@ __global__ void __launch_bounds__(kPairsPerBlock) route_scatter_kernel(const int
                                                                        Workspace ws) {
   __shared__ unsigned short s_cnt[kWarpsPerRouteBlock][kMaxE];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  pdl_launch_dependents();
   for (int i = tid; i < kWarpsPerRouteBlock * E; i += blockDim.x) s_cnt[i / E][i % E] = 0;
   __syncthreads();
   pdl_wait();
+  pdl_launch_dependents();  // after the wait: a kernel downstream may then read, before its own wait, what the kernel before this one wrote
   const int p = blockIdx.x * kPairsPerBlock + tid;
   const int e = (p < P) ? ids[p] : -1;
   const bool valid = (p < P) && e >= 0 && e < E;
