@@ -85,7 +85,12 @@ struct Cfg2 {
   static constexpr int kATiles = (KIND == 0) ? 2 : 1;
   static constexpr int kBRows = BN / 2;                 // token rows staged by each CTA
   static constexpr int kBBytes = kBRows * kBK * 2;
-  static constexpr int kStageBytes = kATiles * kABytes2 + kBBytes;
+  // The down GEMM has one weight tile per stage and half as many MMAs per K block as the
+  // gate/up GEMM, so the fixed cost of a pipeline step (barrier wait, fence, commit) weighs
+  // twice as much there: its stages hold two K blocks (two 64-wide sub-tiles per operand).
+  static constexpr int kSub = (KIND == 1) ? 2 : 1;
+  static constexpr int kSubBytes = kATiles * kABytes2 + kBBytes;
+  static constexpr int kStageBytes = kSub * kSubBytes;
   static constexpr int kAccCols = kATiles * BN;
   static constexpr int kNumAcc = (2 * kAccCols <= 512) ? 2 : 1;
   static constexpr int kTmemCols = (kNumAcc * kAccCols <= 256) ? 256 : 512;
@@ -101,7 +106,7 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
   const int K = (KIND == 0) ? a.H : a.I;
   const int MROWS = (KIND == 0) ? 2 * a.I : a.H;
   const int MT2 = ((KIND == 0) ? a.I : a.H) / (2 * kTileM);  // weight-tile PAIRS per expert
-  const int KB = K / kBK;
+  const int KB = K / (kBK * C::kSub);  // pipeline steps per item
   const int E = a.E;
   const uint32_t rank = cluster_ctarank();
   const int cluster_id = blockIdx.x >> 1;
@@ -172,8 +177,12 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
           const uint32_t full_leader = map_to_cta(bar_full + 8u * kb, 0);
           const uint32_t sa = tiles_base + kb * C::kStageBytes;
           if (rank == 0) mbar_arrive_expect_tx(bar_full + 8u * kb, 2u * C::kStageBytes);  // both CTAs' bytes, activations included
-          tma_load_2d_pair(sa, tmap_w, full_leader, kb * kBK, row_a);
-          if (KIND == 0) tma_load_2d_pair(sa + kABytes2, tmap_w, full_leader, kb * kBK, row_a + a.I);
+          for (int u = 0; u < C::kSub; ++u) {
+            const uint32_t su = sa + u * C::kSubBytes;
+            const int kx = (kb * C::kSub + u) * kBK;
+            tma_load_2d_pair(su, tmap_w, full_leader, kx, row_a);
+            if (KIND == 0) tma_load_2d_pair(su + kABytes2, tmap_w, full_leader, kx, row_a + a.I);
+          }
         }
       }
       pdl_wait();
@@ -195,10 +204,16 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
               break;
             }
             if (rank == 0) mbar_arrive_expect_tx(bar_full + 8u * s, 2u * C::kStageBytes);  // both CTAs' bytes
-            tma_load_2d_pair(sa, tmap_w, full_leader, kb * kBK, row_a);
-            if (KIND == 0) tma_load_2d_pair(sa + kABytes2, tmap_w, full_leader, kb * kBK, row_a + a.I);
+            for (int u = 0; u < C::kSub; ++u) {
+              const uint32_t su = sa + u * C::kSubBytes;
+              const int kx = (kb * C::kSub + u) * kBK;
+              tma_load_2d_pair(su, tmap_w, full_leader, kx, row_a);
+              if (KIND == 0) tma_load_2d_pair(su + kABytes2, tmap_w, full_leader, kx, row_a + a.I);
+            }
           }
-          tma_load_2d_pair(sa + C::kATiles * kABytes2, tmap_act, full_leader, kb * kBK, row_b);
+          for (int u = 0; u < C::kSub; ++u)
+            tma_load_2d_pair(sa + u * C::kSubBytes + C::kATiles * kABytes2, tmap_act, full_leader,
+                             (kb * C::kSub + u) * kBK, row_b);
         }
       }
       (void)ok;
@@ -230,10 +245,14 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
           const uint64_t da1 = umma_desc_sw128(sa + kABytes2);
           const uint64_t db = umma_desc_sw128(sa + C::kATiles * kABytes2);
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) {
-            const uint32_t acc = (kb | k) ? 1u : 0u;
-            umma_bf16_pair(d0, da0 + 2u * k, db + 2u * k, idesc, acc);
-            if (KIND == 0) umma_bf16_pair(d0 + BN, da1 + 2u * k, db + 2u * k, idesc, acc);
+          for (int u = 0; u < C::kSub; ++u) {
+            const uint32_t uo = static_cast<uint32_t>(u) * (C::kSubBytes >> 4);  // next sub-tile, in 16-byte units
+#pragma unroll
+            for (int k = 0; k < kBK / 16; ++k) {
+              const uint32_t acc = (kb | u | k) ? 1u : 0u;
+              umma_bf16_pair(d0, da0 + uo + 2u * k, db + uo + 2u * k, idesc, acc);
+              if (KIND == 0) umma_bf16_pair(d0 + BN, da1 + uo + 2u * k, db + uo + 2u * k, idesc, acc);
+            }
           }
           umma_commit_pair(bar_empty + 8u * s);
         }
