@@ -16,7 +16,11 @@ template <int KIND, int BN, int STAGES>
 struct Cfg {
   static constexpr int kATiles = (KIND == 0) ? 2 : 1;
   static constexpr int kBBytes = BN * kBK * 2;
-  static constexpr int kStageBytes = kATiles * kABytes + kBBytes;
+  // Stages of the wide down GEMM hold two K blocks: with one weight tile per stage its MMAs are
+  // few per pipeline step, and the step's fixed cost (barrier wait, fence, commit) showed.
+  static constexpr int kSub = (KIND == 1 && BN == 128) ? 2 : 1;
+  static constexpr int kSubBytes = kATiles * kABytes + kBBytes;
+  static constexpr int kStageBytes = kSub * kSubBytes;
   static constexpr int kAccCols = kATiles * BN;
   static constexpr int kNumAcc = (2 * kAccCols <= 512) ? 2 : 1;
   static constexpr int kTmemCols = (kNumAcc * kAccCols <= 32)    ? 32
@@ -37,7 +41,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
   const int K = (KIND == 0) ? a.H : a.I;
   const int MROWS = (KIND == 0) ? 2 * a.I : a.H;  // weight rows per expert in the [E*rows, K] view
   const int MT = ((KIND == 0) ? a.I : a.H) / kTileM;
-  const int KB = K / kBK;
+  const int KB = K / (kBK * C::kSub);  // pipeline steps per item
   const int E = a.E;
 
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -108,8 +112,11 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
           const uint32_t full = bar_full + 8u * kb;
           const uint32_t sa = tiles_base + kb * C::kStageBytes;
           mbar_arrive_expect_tx(full, C::kStageBytes);  // the activations' bytes follow after the wait
-          tma_load_2d(sa, tmap_w, full, kb * kBK, row_a);
-          if (KIND == 0) tma_load_2d(sa + kABytes, tmap_w, full, kb * kBK, row_a + a.I);
+          for (int u = 0; u < C::kSub; ++u) {
+            const int kx = (kb * C::kSub + u) * kBK;
+            tma_load_2d(sa + u * C::kSubBytes, tmap_w, full, kx, row_a);
+            if (KIND == 0) tma_load_2d(sa + u * C::kSubBytes + kABytes, tmap_w, full, kx, row_a + a.I);
+          }
         }
       }
       pdl_wait();
@@ -128,10 +135,14 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
               break;
             }
             mbar_arrive_expect_tx(full, C::kStageBytes);
-            tma_load_2d(sa, tmap_w, full, kb * kBK, row_a);
-            if (KIND == 0) tma_load_2d(sa + kABytes, tmap_w, full, kb * kBK, row_a + a.I);
+            for (int u = 0; u < C::kSub; ++u) {
+              const int kx = (kb * C::kSub + u) * kBK;
+              tma_load_2d(sa + u * C::kSubBytes, tmap_w, full, kx, row_a);
+              if (KIND == 0) tma_load_2d(sa + u * C::kSubBytes + kABytes, tmap_w, full, kx, row_a + a.I);
+            }
           }
-          tma_load_2d(sa + C::kATiles * kABytes, tmap_act, full, kb * kBK, item.q0);
+          for (int u = 0; u < C::kSub; ++u)
+            tma_load_2d(sa + u * C::kSubBytes + C::kATiles * kABytes, tmap_act, full, (kb * C::kSub + u) * kBK, item.q0);
         }
       }
       if (!ok) {  // drain what is still in flight so no copy lands after the CTA has gone
@@ -171,13 +182,17 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
           const uint64_t da1 = umma_desc_sw128(sa + kABytes);
           const uint64_t db = umma_desc_sw128(sa + C::kATiles * kABytes);
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) {
-            const uint32_t acc = (kb | k) ? 1u : 0u;
-            umma_bf16(d0, da0 + 2u * k, db + 2u * k, idesc, acc);  // +32 bytes per K=16 step
-            if (KIND == 0) umma_bf16(d0 + BN, da1 + 2u * k, db + 2u * k, idesc, acc);
-            if (kHalfM) {  // rows 64..127 of the weight tile: +64 rows * 128 B in shared memory, +16 TMEM lanes
-              umma_bf16(d0 + (16u << 16), da0 + 512u + 2u * k, db + 2u * k, idesc, acc);
-              if (KIND == 0) umma_bf16(d0 + BN + (16u << 16), da1 + 512u + 2u * k, db + 2u * k, idesc, acc);
+          for (int u = 0; u < C::kSub; ++u) {
+            const uint64_t uo = static_cast<uint64_t>(u) * (C::kSubBytes >> 4);  // next sub-tile, in 16-byte units
+#pragma unroll
+            for (int k = 0; k < kBK / 16; ++k) {
+              const uint32_t acc = (kb | u | k) ? 1u : 0u;
+              umma_bf16(d0, da0 + uo + 2u * k, db + uo + 2u * k, idesc, acc);  // +32 bytes per K=16 step
+              if (KIND == 0) umma_bf16(d0 + BN, da1 + uo + 2u * k, db + uo + 2u * k, idesc, acc);
+              if (kHalfM) {  // rows 64..127 of the weight tile: +64 rows * 128 B in shared memory, +16 TMEM lanes
+                umma_bf16(d0 + (16u << 16), da0 + 512u + 2u * k, db + 2u * k, idesc, acc);
+                if (KIND == 0) umma_bf16(d0 + BN + (16u << 16), da1 + 512u + 2u * k, db + 2u * k, idesc, acc);
+              }
             }
           }
           umma_commit(bar_empty + 8u * s);  // stage is free once these MMAs have read it
