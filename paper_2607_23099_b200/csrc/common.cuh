@@ -59,7 +59,7 @@ constexpr int kNumVariants = 8;
 // id 7: the narrowest tile, N = 8, which bf16 MMAs only offer with M = 64 (two per 128-row weight tile)
 __host__ __device__ constexpr VariantDesc variant_desc(int v) {
   constexpr VariantDesc t[kNumVariants] = {
-      {16, 128, 1, 6, 10}, {32, 128, 1, 5, 10}, {64, 128, 1, 5, 8}, {128, 128, 1, 4, 3}, {256, 128, 1, 3, 4},
+      {16, 128, 1, 6, 10}, {32, 128, 1, 5, 10}, {64, 128, 1, 5, 4}, {128, 128, 1, 4, 3}, {256, 128, 1, 3, 4},
       {128, 256, 2, 5, 4}, {256, 256, 2, 4, 3}, {8, 64, 1, 6, 10}};
   return t[v];
 }

@@ -16,9 +16,11 @@ template <int KIND, int BN, int STAGES>
 struct Cfg {
   static constexpr int kATiles = (KIND == 0) ? 2 : 1;
   static constexpr int kBBytes = BN * kBK * 2;
-  // Stages of the wide down GEMM hold two K blocks: with one weight tile per stage its MMAs are
-  // few per pipeline step, and the step's fixed cost (barrier wait, fence, commit) showed.
-  static constexpr int kSub = (KIND == 1 && BN == 128) ? 2 : 1;
+  // Stages of the N = 64 and N = 128 down GEMMs hold two K blocks: with one weight tile per stage
+  // their MMAs are few per pipeline step, and the step's fixed cost (barrier wait, fence, commit:
+  // some 230 cycles) showed.  The narrow tiles keep one K block per stage (they stream from HBM
+  // and want the finer stages); N = 256 would be left with two stages.
+  static constexpr int kSub = (KIND == 1 && (BN == 64 || BN == 128)) ? 2 : 1;
   static constexpr int kSubBytes = kATiles * kABytes + kBBytes;
   static constexpr int kStageBytes = kSub * kSubBytes;
   static constexpr int kAccCols = kATiles * BN;
