@@ -361,6 +361,14 @@ def dispatch_overhead(m, d, w13, w2, device, reps=30):
     w = WORKLOAD
     stream = torch.cuda.current_stream()
     out = {}
+    # A bucket whose table entries all name one variant needs no selection at all (the host knows
+    # it), so the mechanisms are compared under the cost-model selector, which always decides on
+    # the device among all variants.
+    try:
+        m.set_selector_mode(d.MODE_COST)
+        out["selector_mode"] = "cost model (forces a device-side decision)"
+    except d.DamoeError:
+        out["selector_mode"] = "built-in cost model (no table loaded)"
     for T in (1, 8):
         ids, wts, _ = di.routing_batch(4242 + T, T, w["k"], w["E"], 1.0)
         x = di.activations(4242 + T, T, w["H"], device)
@@ -392,6 +400,10 @@ def dispatch_overhead(m, d, w13, w2, device, reps=30):
         row["auto_graph_switch_us"] = timed(d.VARIANT_AUTO)
         m.set_dispatch(d.DISPATCH_BRANCH)
         out[f"T{T}"] = row
+    try:
+        m.set_selector_mode(d.MODE_EFFEXP_BINS)
+    except d.DamoeError:
+        pass
     out["microbench_us"] = {k: round(v, 2) for k, v in d.dispatch_microbench(200, device.index or 0).items()}
     return out
 

@@ -18,6 +18,8 @@ struct TableBucket {
   int n_bins = 0;
   uint64_t bin_den = 1;
   size_t off_ex = 0, off_exv = 0, off_bnum = 0, off_binv = 0, off_cost = 0;  // byte offsets into the device blob
+  // variants this bucket's entries can select, as bit masks: [0] exemplars, [1] Effective-Experts bins
+  uint32_t cand_ex = 0, cand_bins = 0;
 };
 
 struct damoe_ctx {
@@ -153,8 +155,9 @@ constexpr int kDefaultStaticVariant = 2;
 
 // Fills the selector arguments for this call; returns the host-known variant (>= 0) when the
 // choice does not depend on the routing, else -1.
-int make_selector(const damoe_ctx* c, int T, int variant, SelectorArgs* sel) {
+int make_selector(const damoe_ctx* c, int T, int variant, SelectorArgs* sel, uint32_t* candidates = nullptr) {
   memset(sel, 0, sizeof(*sel));
+  if (candidates) *candidates = ~0u;
   sel->forced = -1;
   sel->mode = DAMOE_MODE_COST;
   sel->cost = c->default_cost;
@@ -174,6 +177,17 @@ int make_selector(const damoe_ctx* c, int T, int variant, SelectorArgs* sel) {
     sel->bin_den = b->bin_den;
     sel->bin_variant = reinterpret_cast<const int32_t*>(c->table_blob + b->off_binv);
     sel->cost = reinterpret_cast<const int64_t*>(c->table_blob + b->off_cost);
+    // The host knows which variants the bucket's entries name.  If it is a single one there is
+    // nothing to select (the call then costs what a static choice costs); otherwise the set tells
+    // the launcher whether the branching kernel has to hold the CTA-pair variants.
+    const uint32_t cand = c->table_mode == DAMOE_MODE_EXEMPLAR ? b->cand_ex
+                          : c->table_mode == DAMOE_MODE_EFFEXP_BINS ? b->cand_bins : ~0u;
+    if (candidates) *candidates = cand;
+    if (cand != 0 && (cand & (cand - 1)) == 0) {
+      int v = 0;
+      while (!((cand >> v) & 1u)) ++v;
+      sel->forced = v;
+    }
   }
   return sel->forced;
 }
@@ -546,6 +560,8 @@ int damoe_load_tuning_table(damoe_ctx* c, const void* bytes, size_t nbytes) {
       if (cost[t] < 0 || cost[t] > (1ll << 36)) return fail(c, DAMOE_ERR_TABLE_FORMAT, "cost out of range in bucket %u", i);
     for (int v = 0; v < kNumVariants; ++v)
       if (!c->variant_ok(v)) cost[v] = 1ll << 36;  // variants this context cannot run
+    for (int32_t v : exv) b.cand_ex |= 1u << v;
+    for (int32_t v : binv) b.cand_bins |= 1u << v;
     b.off_ex = put(ex.data(), ex.size() * 4);
     b.off_exv = put(exv.data(), exv.size() * 4);
     b.off_bnum = put(bnum.data(), bnum.size() * 8);
@@ -623,7 +639,8 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
 #define DAMOE_MARK(i) \
   if (ev) DAMOE_CUDA(c, cudaEventRecord(ev[i], st))
   SelectorArgs sel;
-  const int known = make_selector(c, T, variant, &sel);
+  uint32_t candidates = ~0u;
+  const int known = make_selector(c, T, variant, &sel, &candidates);
   LaunchPack pack;
   build_pack(c, &pack);
   if (known < 0 && c->dispatch == DAMOE_DISPATCH_GRAPH_SWITCH)
@@ -649,13 +666,15 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
     DAMOE_MARK(3);
     DAMOE_CUDA(c, launch_gemm8(1, -1, false, pack.m2, pack.g2, c->sm_count, st));
   } else {
-    // one persistent kernel per GEMM that branches on the variant id; when the CTA-pair variants
-    // exist it is launched as clusters of two so that it can hold the whole family
-    static const bool exp_1cta = getenv("DAMOE_EXP_BRANCH_1CTA") != nullptr;
-    if (c->pairs_ok && !exp_1cta) DAMOE_CUDA(c, launch_gemm2cta(0, -2, false, pack.m13, pack.ga, c->sm_count, st));
+    // one persistent kernel per GEMM that branches on the variant id; when the bucket's entries
+    // can name a CTA-pair variant it is launched as clusters of two so that it holds the whole
+    // family, otherwise as plain CTAs (a few microseconds cheaper to launch)
+    constexpr uint32_t kPairBits = (1u << 5) | (1u << 6);
+    const bool with_pairs = c->pairs_ok && (candidates & kPairBits) != 0;
+    if (with_pairs) DAMOE_CUDA(c, launch_gemm2cta(0, -2, false, pack.m13, pack.ga, c->sm_count, st));
     else DAMOE_CUDA(c, launch_gemm(0, -1, false, pack.m13, pack.ga, c->sm_count, st));
     DAMOE_MARK(3);
-    if (c->pairs_ok && !exp_1cta) DAMOE_CUDA(c, launch_gemm2cta(1, -2, false, pack.m2, pack.ga, c->sm_count, st));
+    if (with_pairs) DAMOE_CUDA(c, launch_gemm2cta(1, -2, false, pack.m2, pack.ga, c->sm_count, st));
     else DAMOE_CUDA(c, launch_gemm(1, -1, false, pack.m2, pack.ga, c->sm_count, st));
   }
   DAMOE_MARK(4);

@@ -57,6 +57,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     default:  // no such variant: still order the kernels after this one behind the kernel before it
       pdl_wait();
       pdl_launch_dependents();
+      if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DAMOE_STATUS_BAD_VARIANT);  // nothing was computed
       break;
   }
 }

@@ -352,6 +352,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
     default:  // no such variant: still order the kernels after this one behind the kernel before it
       pdl_wait();
       pdl_launch_dependents();
+      if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DAMOE_STATUS_BAD_VARIANT);  // nothing was computed
       break;
   }
 }

@@ -149,6 +149,11 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
     if (tid < sel.n_exemplars) s_exv[tid] = sel.ex_variant[tid];
   } else if (select && sel.mode == DAMOE_MODE_COST) {
     if (tid < 4 * kNumVariants) s_cost[tid] = sel.cost[tid];
+  } else if (select && sel.mode == DAMOE_MODE_EFFEXP_BINS) {
+    // thresholds and variants of the bins (at most 64): one parallel load here instead of a
+    // chain of dependent global loads in the selector's single thread
+    if (tid < sel.n_bins) s_exv[tid] = sel.bin_variant[tid];
+    if (tid + 1 < sel.n_bins) s_score[tid] = static_cast<long long>(sel.bin_num[tid]);
   }
   if (FUSED) {
     for (int e = tid; e < E; e += kScanThreads) s_hist[e] = 0;
@@ -343,8 +348,8 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(int32_t* __res
       const unsigned long long a = s_red[0][0], b = s_red[1][0];
       int r = 0;
       for (int i = 0; i + 1 < sel.n_bins; ++i)
-        if (a * a * sel.bin_den >= sel.bin_num[i] * b) ++r;
-      chosen = sel.bin_variant[r];
+        if (a * a * sel.bin_den >= static_cast<unsigned long long>(s_score[i]) * b) ++r;
+      chosen = s_exv[r];
     }
   } else {  // DAMOE_MODE_COST
     if (tid < kNumVariants) {
