@@ -84,7 +84,7 @@ def table_path(w):
 # activated experts of the captured cell (profiles/gemm_gate_up_small_E32_T8_ncu_full.md):
 # bytes per activated expert.  The capture is of the reduced case; traffic grows in proportion
 # to the activated experts, so bench scales it by its own cells' counts.
-NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 = 59.01e6
+NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 = 58.98e6
 
 
 def peaks():
@@ -537,8 +537,8 @@ def run_ours(args):
     traffic = None
     if not fp8 and not is_trace and "grid" not in w:
         traffic = round(NCU_TRAFFIC_PER_ACTIVE_EXPERT_W13 * statistics.mean(c["active"] for c in rec_cells))
-    kernel_name = ("gemm8_branch_kernel<0>" if fp8 else "gemm2_branch_kernel<0>") + \
-        " (grouped gate/up GEMM + SwiGLU, branching on the device-side variant id)"
+    kernel_name = ("gemm8_branch_kernel<0>" if fp8 else "gemm_fixed_kernel<0, v> / gemm_branch_kernel<0> / gemm2_branch_kernel<0>") + \
+        " (grouped gate/up GEMM + SwiGLU; the fixed-variant kernel where the table bucket names one variant, else the kernel branching on the device-side variant id)"
     share = {k: round(stage[k] / max(1e-9, sum(stage[s] for s in m.STAGES)), 4) for k in m.STAGES}
     # the gate/up GEMM's own two bounds: its bytes over HBM, its useful flops over the tensor peak
     w13_flops = statistics.mean(float(c["hist"].sum()) * 4 * w["H"] * w["I"] for c in rec_cells)
