@@ -12,8 +12,12 @@
 // epilogue: four warps per TMEM lane quadrant (two for the narrowest tile), each owning a group of
 // N_v / 4 token columns.  Every K block has to pass through all epilogue warps, so the promotion
 // rate is set by the work of ONE warp per K block; spreading the columns over four groups (and
-// four warps per scheduler to hide the TMEM-load and shuffle latencies) is what keeps it from
-// throttling the MMAs, and it keeps the register accumulators at N_v / 2 floats per thread.
+// four warps per scheduler to hide the TMEM-load latency) is what keeps it from throttling the
+// MMAs, and it keeps the register accumulators at N_v / 2 floats per thread (576 threads leave
+// 96 registers each).  Per K block a warp writes the products  act_scale[col] * w_scale  of its
+// columns to a small shared-memory table (one lane per column) and the promotion reads two
+// columns' products with one 16-byte broadcast load: one FMA per element.  The scales themselves
+// are fetched from global memory two K blocks ahead.
 //
 // KIND 0 (gate/up): a = silu(g) * u, h_b = bf16(a); the 128 channels of the weight tile are
 //   exactly one 1x128 scale group of h, so the group amax is a reduction over the tile's 128
@@ -31,7 +35,8 @@ namespace {
 
 constexpr int kThreads8 = 576;  // 2 + 16 warps
 constexpr int kABytes8 = kTileM * kBK8;  // 128 rows x 128 one-byte elements
-constexpr int kTailBytes8 = 2 * (kMaxE + 1) * 4 + 512 + 2 * 4 * 128 * 4;  // + amax exchange, double-buffered [2][4 quadrants][BN <= 128]
+constexpr int kTailBytes8 = 2 * (kMaxE + 1) * 4 + 512 + 2 * 4 * 128 * 4   // + amax exchange, double-buffered [2][4 quadrants][BN <= 128]
+                            + 16 * 2 * 32 * 8 + 16;                  // + per-warp scale products, double-buffered [16 warps][2][CW <= 32] float2
 
 __device__ __forceinline__ void umma_fp8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                          uint32_t accumulate) {
@@ -114,6 +119,8 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
   constexpr int NP = C::kNumPartials;
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   float* s_amax = reinterpret_cast<float*>(s_tmem + 2);  // [2 buffers][4 quadrants][BN]
+  // per epilogue warp: the K block's scale products per token column, {act*w_gate, act*w_up}, 16-byte aligned
+  float2* s_scale = reinterpret_cast<float2*>((reinterpret_cast<uintptr_t>(s_amax + 2 * 4 * 128) + 15) & ~uintptr_t(15));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -237,16 +244,37 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
         for (int j = 0; j < CW; ++j) acc_u[j] = 0.f;
       }
       bool ok = true;
+      // The scales of a K block come from global memory; they are requested two K blocks ahead so
+      // that their latency never sits between an MMA's completion and its promotion.
+      const float* xs_base = a.act_scale_T + item.q0 + col0 + lane;
+      const bool has_col = lane < CW && col0 + lane < item.valid;
+      auto fetch = [&](int kb, float& sx, float& sg, float& su) {
+        sx = 0.f;
+        sg = 0.f;
+        su = 0.f;
+        if (kb < KB) {
+          if (has_col) sx = __ldg(xs_base + static_cast<size_t>(kb) * a.max_P);
+          sg = __ldg(wg + kb);
+          if (KIND == 0) su = __ldg(wu + kb);
+        }
+      };
+      float sx_a, sg_a, su_a, sx_b, sg_b, su_b;
+      fetch(0, sx_a, sg_a, su_a);
+      fetch(1, sx_b, sg_b, su_b);
       for (int kb = 0; kb < KB; ++kb, ++it) {
         const int pb = it % NP;
         const uint32_t pph = (it / NP) & 1;
-        // this lane's share of the activation scales of the K block: lane l holds column col0+l (and +32)
-        const float* xs = a.act_scale_T + static_cast<size_t>(kb) * a.max_P + item.q0 + col0;
-        float sx0 = 0.f, sx1 = 0.f;
-        if (lane < CW && col0 + lane < item.valid) sx0 = __ldg(xs + lane);
-        if (CW > 32 && col0 + 32 + lane < item.valid) sx1 = __ldg(xs + 32 + lane);
-        const float swg = __ldg(wg + kb);
-        const float swu = (KIND == 0) ? __ldg(wu + kb) : 0.f;
+        // Lane l fetches the activation scale of column col0+l and writes the products with the two
+        // weight-block scales to the warp's table; the promotion below then reads two columns'
+        // products with one 16-byte broadcast load and spends one FMA per element.
+        const float sx0 = sx_a, swg = sg_a, swu = su_a;
+        sx_a = sx_b;
+        sg_a = sg_b;
+        su_a = su_b;
+        fetch(kb + 2, sx_b, sg_b, su_b);
+        float2* sc = s_scale + (ew * 2 + (kb & 1)) * 32;
+        if (lane < CW) sc[lane] = make_float2(sx0 * swg, sx0 * swu);
+        __syncwarp();
         if (!mbar_wait(bar_pfull + 8u * pb, pph, s_abort)) {
           ok = false;
           break;
@@ -256,8 +284,10 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
         // Only the 16-column (8 for the narrowest tile) chunks that hold valid tokens are promoted.
         // All TMEM loads of a group of up to 32 columns (gate and up) are issued before the one
         // wait, so their latency is paid once per group instead of once per chunk.
-        constexpr int CH = CW < 16 ? CW : 16;
-        constexpr int GW = CW < 32 ? CW : 32;   // columns per group
+        // The widest gate/up tile keeps 64 accumulators per thread, so it reads the partials in
+        // pieces of 8 columns (16 values in flight) to stay within the register budget.
+        constexpr int CH = (CW < 16 || (KIND == 0 && CW == 32)) ? 8 : 16;
+        constexpr int GW = CH;   // columns per group: loaded, waited for and promoted together
 #pragma unroll
         for (int g0 = 0; g0 < CW; g0 += GW) {
           if (col0 + g0 < item.valid) {  // warp-uniform
@@ -279,11 +309,15 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
             for (int c = 0; c < GW; c += CH) {
               if (col0 + g0 + c < item.valid) {
 #pragma unroll
-                for (int j = 0; j < CH; ++j) {
+                for (int j = 0; j < CH; j += 2) {
                   const int col = g0 + c + j;
-                  const float sx = __shfl_sync(0xffffffffu, (col < 32) ? sx0 : sx1, col & 31);
-                  acc_g[col] = fmaf(__uint_as_float(pg[c + j]), sx * swg, acc_g[col]);
-                  if constexpr (KIND == 0) acc_u[col] = fmaf(__uint_as_float(pu[c + j]), sx * swu, acc_u[col]);
+                  const float4 q = *reinterpret_cast<const float4*>(sc + col);  // {g, u} of col and col + 1
+                  acc_g[col] = fmaf(__uint_as_float(pg[c + j]), q.x, acc_g[col]);
+                  acc_g[col + 1] = fmaf(__uint_as_float(pg[c + j + 1]), q.z, acc_g[col + 1]);
+                  if constexpr (KIND == 0) {
+                    acc_u[col] = fmaf(__uint_as_float(pu[c + j]), q.y, acc_u[col]);
+                    acc_u[col + 1] = fmaf(__uint_as_float(pu[c + j + 1]), q.w, acc_u[col + 1]);
+                  }
                 }
               }
             }
@@ -299,12 +333,12 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
         // The exchange buffer alternates per item; a warp can only reach item i+2 after all four
         // warps of its half have arrived at item i+1's exchange, i.e. after they read item i's.
         float* xa = s_amax + (item_i & 1) * 4 * BN;
-        float hb[CW];
+        // h_b takes the place of the gate accumulator (no second array of CW registers)
 #pragma unroll
         for (int j = 0; j < CW; ++j) {
           if (col0 + j < item.valid) {  // warp-uniform
-            hb[j] = __bfloat162float(__float2bfloat16_rn(silu_mul(acc_g[j], acc_u[j])));
-            const unsigned m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(hb[j])));
+            acc_g[j] = __bfloat162float(__float2bfloat16_rn(silu_mul(acc_g[j], acc_u[j])));
+            const unsigned m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(acc_g[j])));
             if (lane == 0) xa[quad * BN + col0 + j] = __uint_as_float(m);
           }
         }
@@ -317,7 +351,7 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
           if (n < item.valid) {
             const float amax = fmaxf(fmaxf(xa[0 * BN + n], xa[1 * BN + n]), fmaxf(xa[2 * BN + n], xa[3 * BN + n]));
             const float sc = (amax == 0.f) ? 1.0f : __fdiv_rn(amax, 448.0f);
-            const uint8_t code = static_cast<uint8_t>(__nv_cvt_float_to_fp8(__fdiv_rn(hb[j], sc), __NV_SATFINITE, __NV_E4M3));
+            const uint8_t code = static_cast<uint8_t>(__nv_cvt_float_to_fp8(__fdiv_rn(acc_g[j], sc), __NV_SATFINITE, __NV_E4M3));
             a.hq[static_cast<size_t>(item.q0 + n) * a.I + ch] = code;
             if (quad == 0 && lane == 0) a.hs_T[static_cast<size_t>(item.m_tile) * a.max_P + item.q0 + n] = sc;
           }
