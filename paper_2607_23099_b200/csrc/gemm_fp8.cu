@@ -12,12 +12,12 @@
 // epilogue: four warps per TMEM lane quadrant (two for the narrowest tile), each owning a group of
 // N_v / 4 token columns.  Every K block has to pass through all epilogue warps, so the promotion
 // rate is set by the work of ONE warp per K block; spreading the columns over four groups (and
-// four warps per scheduler to hide the TMEM-load latency) is what keeps it from throttling the
-// MMAs, and it keeps the register accumulators at N_v / 2 floats per thread (576 threads leave
-// 96 registers each).  Per K block a warp writes the products  act_scale[col] * w_scale  of its
-// columns to a small shared-memory table (one lane per column) and the promotion reads two
-// columns' products with one 16-byte broadcast load: one FMA per element.  The scales themselves
-// are fetched from global memory two K blocks ahead.
+// four warps per scheduler to hide the TMEM-load and shuffle latencies) is what keeps it from
+// throttling the MMAs, and it keeps the register accumulators at N_v / 2 floats per thread (576
+// threads leave 96 registers each).  A lane holds the activation scale of one column and the
+// promotion broadcasts it with a shuffle; a shared-memory table of the scale products (one FMA
+// per element instead of shuffle + multiply + FMA) measured 2-4 % slower.  The scales are
+// fetched from global memory two K blocks ahead.
 //
 // KIND 0 (gate/up): a = silu(g) * u, h_b = bf16(a); the 128 channels of the weight tile are
 //   exactly one 1x128 scale group of h, so the group amax is a reduction over the tile's 128
@@ -35,8 +35,7 @@ namespace {
 
 constexpr int kThreads8 = 576;  // 2 + 16 warps
 constexpr int kABytes8 = kTileM * kBK8;  // 128 rows x 128 one-byte elements
-constexpr int kTailBytes8 = 2 * (kMaxE + 1) * 4 + 512 + 2 * 4 * 128 * 4   // + amax exchange, double-buffered [2][4 quadrants][BN <= 128]
-                            + 16 * 2 * 32 * 8 + 16;                  // + per-warp scale products, double-buffered [16 warps][2][CW <= 32] float2
+constexpr int kTailBytes8 = 2 * (kMaxE + 1) * 4 + 512 + 2 * 4 * 128 * 4;  // + amax exchange, double-buffered [2][4 quadrants][BN <= 128]
 
 __device__ __forceinline__ void umma_fp8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                          uint32_t accumulate) {
@@ -119,8 +118,6 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
   constexpr int NP = C::kNumPartials;
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   float* s_amax = reinterpret_cast<float*>(s_tmem + 2);  // [2 buffers][4 quadrants][BN]
-  // per epilogue warp: the K block's scale products per token column, {act*w_gate, act*w_up}, 16-byte aligned
-  float2* s_scale = reinterpret_cast<float2*>((reinterpret_cast<uintptr_t>(s_amax + 2 * 4 * 128) + 15) & ~uintptr_t(15));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -249,9 +246,7 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
       const float* xs_base = a.act_scale_T + item.q0 + col0 + lane;
       const bool has_col = lane < CW && col0 + lane < item.valid;
       auto fetch = [&](int kb, float& sx, float& sg, float& su) {
-        sx = 0.f;
-        sg = 0.f;
-        su = 0.f;
+        sx = 0.f; sg = 0.f; su = 0.f;
         if (kb < KB) {
           if (has_col) sx = __ldg(xs_base + static_cast<size_t>(kb) * a.max_P);
           sg = __ldg(wg + kb);
@@ -264,17 +259,9 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
       for (int kb = 0; kb < KB; ++kb, ++it) {
         const int pb = it % NP;
         const uint32_t pph = (it / NP) & 1;
-        // Lane l fetches the activation scale of column col0+l and writes the products with the two
-        // weight-block scales to the warp's table; the promotion below then reads two columns'
-        // products with one 16-byte broadcast load and spends one FMA per element.
-        const float sx0 = sx_a, swg = sg_a, swu = su_a;
-        sx_a = sx_b;
-        sg_a = sg_b;
-        su_a = su_b;
+        const float sx0 = sx_a, swg = sg_a, swu = su_a, sx1 = 0.f;
+        sx_a = sx_b; sg_a = sg_b; su_a = su_b;
         fetch(kb + 2, sx_b, sg_b, su_b);
-        float2* sc = s_scale + (ew * 2 + (kb & 1)) * 32;
-        if (lane < CW) sc[lane] = make_float2(sx0 * swg, sx0 * swu);
-        __syncwarp();
         if (!mbar_wait(bar_pfull + 8u * pb, pph, s_abort)) {
           ok = false;
           break;
@@ -286,8 +273,9 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
         // wait, so their latency is paid once per group instead of once per chunk.
         // The widest gate/up tile keeps 64 accumulators per thread, so it reads the partials in
         // pieces of 8 columns (16 values in flight) to stay within the register budget.
-        constexpr int CH = (CW < 16 || (KIND == 0 && CW == 32)) ? 8 : 16;
-        constexpr int GW = CH;   // columns per group: loaded, waited for and promoted together
+        constexpr bool kNarrowReads = (KIND == 0 && CW == 32);
+        constexpr int CH = (CW < 16 || kNarrowReads) ? 8 : 16;
+        constexpr int GW = kNarrowReads ? 8 : (CW < 32 ? CW : 32);   // columns per group
 #pragma unroll
         for (int g0 = 0; g0 < CW; g0 += GW) {
           if (col0 + g0 < item.valid) {  // warp-uniform
@@ -309,15 +297,11 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
             for (int c = 0; c < GW; c += CH) {
               if (col0 + g0 + c < item.valid) {
 #pragma unroll
-                for (int j = 0; j < CH; j += 2) {
+                for (int j = 0; j < CH; ++j) {
                   const int col = g0 + c + j;
-                  const float4 q = *reinterpret_cast<const float4*>(sc + col);  // {g, u} of col and col + 1
-                  acc_g[col] = fmaf(__uint_as_float(pg[c + j]), q.x, acc_g[col]);
-                  acc_g[col + 1] = fmaf(__uint_as_float(pg[c + j + 1]), q.z, acc_g[col + 1]);
-                  if constexpr (KIND == 0) {
-                    acc_u[col] = fmaf(__uint_as_float(pu[c + j]), q.y, acc_u[col]);
-                    acc_u[col + 1] = fmaf(__uint_as_float(pu[c + j + 1]), q.w, acc_u[col + 1]);
-                  }
+                  const float sx = __shfl_sync(0xffffffffu, (col < 32) ? sx0 : sx1, col & 31);
+                  acc_g[col] = fmaf(__uint_as_float(pg[c + j]), sx * swg, acc_g[col]);
+                  if constexpr (KIND == 0) acc_u[col] = fmaf(__uint_as_float(pu[c + j]), sx * swu, acc_u[col]);
                 }
               }
             }
