@@ -243,8 +243,6 @@ void build_pack(const damoe_ctx* c, LaunchPack* p) {
   ga.h = c->ws.h;
   ga.y = c->ws.y;
   ga.E = c->E; ga.H = c->H; ga.I = c->I;
-  static const int even = getenv("DAMOE_EVEN_SPLIT") ? atoi(getenv("DAMOE_EVEN_SPLIT")) : 1;
-  ga.even_split = even;
   p->ga = ga;
   GemmArgs8 g13{}, g2{};
   g13.ntile_prefix = g2.ntile_prefix = c->ws.ntile_prefix;
@@ -256,7 +254,6 @@ void build_pack(const damoe_ctx* c, LaunchPack* p) {
   g13.hs_T = g2.hs_T = c->ws.hs_T;
   g13.y = g2.y = c->ws.y;
   g13.E = g2.E = c->E; g13.H = g2.H = c->H; g13.I = g2.I = c->I; g13.max_P = g2.max_P = c->max_P;
-  g13.even_split = g2.even_split = even;
   g13.w_scale = c->w13_scale; g13.act_scale_T = c->ws.xs_T;
   g2.w_scale = c->w2_scale; g2.act_scale_T = c->ws.hs_T;
   p->g13 = g13;

@@ -129,7 +129,6 @@ struct GemmArgs {
   __nv_bfloat16* h;             // gate/up GEMM output [max_P, I]
   float* y;                     // down GEMM output [max_P, H]
   int E, H, I;
-  int even_split;               // split an expert's tokens evenly over its tiles (else N_v, N_v, ..., rest)
 };
 // variant >= 0: launch that variant's kernel; predicated: it exits unless *variant_id == variant.
 // variant == -1: one kernel that branches on *variant_id.
@@ -157,7 +156,6 @@ struct GemmArgs8 {
   float* hs_T;            // gate/up output scales [I/128, max_P]
   float* y;               // down GEMM output [max_P, H]
   int E, H, I, max_P;
-  int even_split;
 };
 cudaError_t launch_gemm8(int kind, int variant, bool predicated, const GemmMaps& maps, const GemmArgs8& args,
                          int sm_count, cudaStream_t stream);

@@ -107,7 +107,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
       // The weights of the first item start streaming before the upstream kernel has finished.
       int n_pre = 0;
       if (static_cast<int>(blockIdx.x) < total) {
-        const Item item = decode_item(blockIdx.x, s_pref, s_off, E, MT, BN, a.even_split);
+        const Item item = decode_item(blockIdx.x, s_pref, s_off, E, MT);
         const int row_a = item.e * MROWS + item.m_tile * kTileM;
         n_pre = KB < STAGES ? KB : STAGES;
         for (int kb = 0; kb < n_pre; ++kb) {
@@ -124,7 +124,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
       pdl_wait();
       pdl_launch_dependents();
       for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
-        const Item item = decode_item(w, s_pref, s_off, E, MT, BN, a.even_split);
+        const Item item = decode_item(w, s_pref, s_off, E, MT);
         const int row_a = item.e * MROWS + item.m_tile * kTileM;
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const int s = it % STAGES;
@@ -161,7 +161,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
       for (int w = blockIdx.x; ok && w < total; w += gridDim.x, ++tile_i) {
         // A ragged last token tile issues narrower MMAs: N is a field of the instruction
         // descriptor, so only ceil16(valid) token columns cost tensor time.
-        const Item item = decode_item(w, s_pref, s_off, E, MT, BN, a.even_split);
+        const Item item = decode_item(w, s_pref, s_off, E, MT);
         const int n_eff = (item.valid + 15) & ~15;
         // N = 8 exists only with M = 64: the 128-row weight tile is then two MMAs, whose
         // accumulator rows land in the lower and the upper 16 lanes of each TMEM lane quadrant
@@ -207,7 +207,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap* tmap_w, const CUten
     const uint32_t lane_base = (warp & 3) * 32;  // the TMEM lane quadrant this warp may read
     int tile_i = 0;
     for (int w = blockIdx.x; w < total; w += gridDim.x, ++tile_i) {
-      const Item item = decode_item(w, s_pref, s_off, E, MT, BN, a.even_split);
+      const Item item = decode_item(w, s_pref, s_off, E, MT);
       const int buf = tile_i % C::kNumAcc;
       const uint32_t aph = (tile_i / C::kNumAcc) & 1;
       if (!mbar_wait(bar_tfull + 8u * buf, aph, s_abort)) break;

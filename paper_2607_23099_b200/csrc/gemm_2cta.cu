@@ -170,7 +170,7 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
       bool ok = true;
       int n_pre = 0;
       if (cluster_id < total) {  // the first item's weights, before the upstream kernel has finished
-        const Item item = decode_item(cluster_id, s_pref, s_off, E, MT2, BN, a.even_split);
+        const Item item = decode_item(cluster_id, s_pref, s_off, E, MT2);
         const int row_a = item.e * MROWS + (2 * item.m_tile + static_cast<int>(rank)) * kTileM;
         n_pre = KB < STAGES ? KB : STAGES;
         for (int kb = 0; kb < n_pre; ++kb) {
@@ -188,7 +188,7 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
       pdl_wait();
       pdl_launch_dependents();
       for (int w = cluster_id; ok && w < total; w += num_clusters) {
-        const Item item = decode_item(w, s_pref, s_off, E, MT2, BN, a.even_split);   // item.m_tile = pair index
+        const Item item = decode_item(w, s_pref, s_off, E, MT2);   // item.m_tile = pair index
         const int n_eff = (item.valid + 15) & ~15;
         const int n_use = n_eff < BN ? n_eff : BN;
         const int row_a = item.e * MROWS + (2 * item.m_tile + static_cast<int>(rank)) * kTileM;
@@ -224,7 +224,7 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
       int it = 0, tile_i = 0;
       bool ok = true;
       for (int w = cluster_id; ok && w < total; w += num_clusters, ++tile_i) {
-        const Item item = decode_item(w, s_pref, s_off, E, MT2, BN, a.even_split);
+        const Item item = decode_item(w, s_pref, s_off, E, MT2);
         const int n_eff = (item.valid + 15) & ~15;
         const uint32_t idesc = umma_idesc_bf16(2 * kTileM, n_eff < BN ? n_eff : BN);
         const int buf = tile_i % C::kNumAcc;
@@ -264,7 +264,7 @@ __device__ __forceinline__ void gemm2_body(const CUtensorMap* tmap_w, const CUte
     const uint32_t lane_base = (warp & 3) * 32;
     int tile_i = 0;
     for (int w = cluster_id; w < total; w += num_clusters, ++tile_i) {
-      const Item item = decode_item(w, s_pref, s_off, E, MT2, BN, a.even_split);
+      const Item item = decode_item(w, s_pref, s_off, E, MT2);
       const int buf = tile_i % C::kNumAcc;
       const uint32_t aph = (tile_i / C::kNumAcc) & 1;
       if (!mbar_wait(bar_tfull + 8u * buf, aph, s_abort)) break;

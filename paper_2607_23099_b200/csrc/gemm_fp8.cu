@@ -160,7 +160,7 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
       int it = 0;
       bool ok = true;
       for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
-        const Item item = decode_item(w, s_pref, s_off, E, MT, BN, a.even_split);
+        const Item item = decode_item(w, s_pref, s_off, E, MT);
         const int row_a = item.e * MROWS + item.m_tile * kTileM;
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const int s = it % STAGES;
@@ -189,7 +189,7 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
       int it = 0;
       bool ok = true;
       for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
-        const Item item = decode_item(w, s_pref, s_off, E, MT, BN, a.even_split);
+        const Item item = decode_item(w, s_pref, s_off, E, MT);
         const int n_eff = (item.valid + 15) & ~15;
         const uint32_t idesc = umma_idesc_e4m3(kTileM, n_eff < BN ? n_eff : BN);
         for (int kb = 0; kb < KB; ++kb, ++it) {
@@ -228,7 +228,7 @@ __device__ __forceinline__ void gemm8_body(const CUtensorMap* tmap_w, const CUte
     const float* wsc = a.w_scale;
     int it = 0, item_i = 0;
     for (int w = blockIdx.x; half < G && w < total; w += gridDim.x, ++item_i) {
-      const Item item = decode_item(w, s_pref, s_off, E, MT, BN, a.even_split);
+      const Item item = decode_item(w, s_pref, s_off, E, MT);
       const int ch = item.m_tile * kTileM + lane_base + lane;
       // weight-scale rows of this item: [expert, row block, K block]
       const float* wg = wsc + (static_cast<size_t>(item.e) * (MROWS / 128) + item.m_tile) * wblocks_k;
