@@ -228,6 +228,16 @@ def routing_batch(seed: int, T: int, k: int, E: int, alpha: float):
     return ids, w, np.exp(log_p)
 
 
+def router_logits(seed: int, T: int, E: int, alpha: float) -> np.ndarray:
+    """Router logits [T, E] float32 whose per-token top-k is a draw of k distinct experts in
+    proportion to p ~ Dirichlet(alpha): log p_e plus independent Gumbel noise (the same model and
+    the same random streams as routing_batch, which keeps the result of the top-k only)."""
+    log_p = dirichlet_log_p(alpha, E, 1, _rng(seed, 1))[0]
+    u = _rng(seed, 2).random(size=(T, E))
+    u = np.clip(u, np.finfo(np.float64).tiny, 1.0 - 2.0 ** -53)
+    return (log_p[None, :] - np.log(-np.log(u))).astype(np.float32)
+
+
 def shard_ids(ids: np.ndarray, E_local: int, shard: int = 0) -> np.ndarray:
     """Expert-parallel view of a global routing: experts [shard*E_local, (shard+1)*E_local) are
     renumbered from 0, every other id becomes -1 (the library skips ids outside [0, E))."""

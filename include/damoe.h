@@ -155,6 +155,34 @@ int damoe_fused_moe(damoe_ctx* ctx, const void* x, const void* w13, const void* 
                     void* out, void* stream);
 
 /*
+ * Router selection, the step upstream of the layer.  The paper measures an "end-to-end
+ * MoE-layer latency" that covers router selection, routing-metadata construction, dispatch
+ * and the fused-MoE execution (Section V); it does not define the gating function, so this
+ * follows the build's configurations: per token the k largest of the E router logits are
+ * selected (equal logits: the lower expert index first; NaN sorts below every number) and the
+ * routing weights are the softmax over the k selected logits.
+ *
+ * logits: dev [T, E] float32 row-major (E of the context).  topk_ids: dev [T, k] int32, written
+ * in order of descending logit.  topk_weights: dev [T, k] float32.  0 <= T <= max_T; T == 0
+ * returns DAMOE_OK and touches nothing.  Enqueues one kernel on `stream`; never synchronises.
+ */
+int damoe_router_topk(damoe_ctx* ctx, const float* logits, int T, int32_t* topk_ids, float* topk_weights,
+                      void* stream);
+
+/*
+ * The layer from router logits: damoe_router_topk into buffers the context owns, then
+ * damoe_fused_moe on them (same `variant` argument, same rules).  This is the call the
+ * end-to-end MoE-layer latency is measured on.  The selected ids and weights can be read back
+ * afterwards with damoe_debug_fetch_routing.
+ */
+int damoe_moe_from_logits(damoe_ctx* ctx, const void* x, const void* w13, const void* w2, const float* logits,
+                          int T, int variant, void* out, void* stream);
+
+/* Test / diagnostic (synchronises): copies the ids [T,k] and weights [T,k] that the last
+ * damoe_moe_from_logits call selected to host memory. */
+int damoe_debug_fetch_routing(damoe_ctx* ctx, int T, int32_t* topk_ids_host, float* topk_weights_host);
+
+/*
  * End-to-end form with the per-step tensors on the HOST: x_host [T,H] bf16, topk_ids_host
  * [T,k] int32, topk_weights_host [T,k] float32 are copied to the device, the layer runs, and
  * out_host [T,H] bf16 is copied back; the call returns after the result has arrived

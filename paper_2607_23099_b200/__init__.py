@@ -27,6 +27,7 @@ EXPORTS = [
     "damoe_fused_moe_host", "damoe_set_fp8_scales", "damoe_load_tuning_table", "damoe_set_dispatch",
     "damoe_variant_count", "damoe_variant_info", "damoe_debug_fetch", "damoe_dispatch_microbench",
     "damoe_set_profiling", "damoe_get_stage_ms", "damoe_route_stats_noalloc", "damoe_set_selector_mode",
+    "damoe_router_topk", "damoe_moe_from_logits", "damoe_debug_fetch_routing",
 ]
 
 
@@ -44,6 +45,9 @@ def _load() -> ctypes.CDLL:
     lib.damoe_route_stats.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     lib.damoe_fused_moe.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
     lib.damoe_fused_moe_host.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
+    lib.damoe_router_topk.argtypes = [vp, vp, i32, vp, vp, vp]
+    lib.damoe_moe_from_logits.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, vp]
+    lib.damoe_debug_fetch_routing.argtypes = [vp, i32, vp, vp]
     lib.damoe_set_fp8_scales.argtypes = [vp, vp, vp, vp]
     lib.damoe_load_tuning_table.argtypes = [vp, ctypes.c_char_p, ctypes.c_size_t]
     lib.damoe_set_dispatch.argtypes = [vp, i32]
@@ -158,6 +162,31 @@ class DAMoE:
         self._check(_lib.damoe_fused_moe(self._ctx, _ptr(x), _ptr(w13), _ptr(w2), _ptr(topk_ids), _ptr(topk_weights),
                                          T, variant, _ptr(out), _stream_ptr(stream)))
         return out
+
+    def router_topk(self, logits, topk_ids=None, topk_weights=None, stream=None):
+        """Router selection: per token the k largest of the E logits and the softmax over them."""
+        T = logits.shape[0]
+        dev = logits.device
+        topk_ids = torch.empty(T, self.k, dtype=torch.int32, device=dev) if topk_ids is None else topk_ids
+        topk_weights = torch.empty(T, self.k, dtype=torch.float32, device=dev) if topk_weights is None else topk_weights
+        self._check(_lib.damoe_router_topk(self._ctx, _ptr(logits), T, _ptr(topk_ids), _ptr(topk_weights),
+                                           _stream_ptr(stream)))
+        return topk_ids, topk_weights
+
+    def moe_from_logits(self, x, w13, w2, logits, variant: int = VARIANT_AUTO, out=None, stream=None):
+        """The layer from router logits (router selection + fused_moe)."""
+        T = x.shape[0]
+        out = torch.empty(T, self.H, dtype=torch.bfloat16, device=x.device) if out is None else out
+        self._check(_lib.damoe_moe_from_logits(self._ctx, _ptr(x), _ptr(w13), _ptr(w2), _ptr(logits), T, variant,
+                                               _ptr(out), _stream_ptr(stream)))
+        return out
+
+    def debug_fetch_routing(self, T: int):
+        """ids and weights selected by the last moe_from_logits call (synchronises)."""
+        ids = torch.empty(T, self.k, dtype=torch.int32)
+        w = torch.empty(T, self.k, dtype=torch.float32)
+        self._check(_lib.damoe_debug_fetch_routing(self._ctx, T, _ptr(ids), _ptr(w)))
+        return ids.numpy(), w.numpy()
 
     def fused_moe_host(self, x_host, w13, w2, topk_ids_host, topk_weights_host, variant: int = VARIANT_AUTO,
                        out_host=None, stream=None):

@@ -681,6 +681,38 @@ int damoe_fused_moe(damoe_ctx* c, const void* x, const void* w13, const void* w2
   return DAMOE_OK;
 }
 
+int damoe_router_topk(damoe_ctx* c, const float* logits, int T, int32_t* topk_ids, float* topk_weights, void* stream) {
+  if (!c) return DAMOE_ERR_INVALID_ARG;
+  if (T == 0) return DAMOE_OK;
+  if (T < 0 || T > c->max_T || !logits || !topk_ids || !topk_weights) return fail(c, DAMOE_ERR_INVALID_ARG, "bad argument");
+  if (c->k > c->E) return fail(c, DAMOE_ERR_INVALID_ARG, "k = %d exceeds E = %d", c->k, c->E);
+  DAMOE_CUDA(c, cudaSetDevice(c->device));
+  DAMOE_CUDA(c, launch_router_topk(logits, T, c->E, c->k, topk_ids, topk_weights, static_cast<cudaStream_t>(stream)));
+  return DAMOE_OK;
+}
+
+int damoe_moe_from_logits(damoe_ctx* c, const void* x, const void* w13, const void* w2, const float* logits, int T,
+                          int variant, void* out, void* stream) {
+  if (!c) return DAMOE_ERR_INVALID_ARG;
+  if (T == 0) return DAMOE_OK;
+  // the staging buffers of the host-buffer entry point double as the context's routing buffers
+  int32_t* ids = static_cast<int32_t*>(c->st_ids);
+  float* wts = static_cast<float*>(c->st_w);
+  const int rc = damoe_router_topk(c, logits, T, ids, wts, stream);
+  if (rc != DAMOE_OK) return rc;
+  return damoe_fused_moe(c, x, w13, w2, ids, wts, T, variant, out, stream);
+}
+
+int damoe_debug_fetch_routing(damoe_ctx* c, int T, int32_t* topk_ids_host, float* topk_weights_host) {
+  if (!c || T < 0 || T > c->max_T) return DAMOE_ERR_INVALID_ARG;
+  DAMOE_CUDA(c, cudaSetDevice(c->device));
+  DAMOE_CUDA(c, cudaDeviceSynchronize());
+  const size_t P = static_cast<size_t>(T) * c->k;
+  if (topk_ids_host) DAMOE_CUDA(c, cudaMemcpy(topk_ids_host, c->st_ids, 4 * P, cudaMemcpyDeviceToHost));
+  if (topk_weights_host) DAMOE_CUDA(c, cudaMemcpy(topk_weights_host, c->st_w, 4 * P, cudaMemcpyDeviceToHost));
+  return DAMOE_OK;
+}
+
 int damoe_fused_moe_host(damoe_ctx* c, const void* x_host, const void* w13, const void* w2,
                          const int32_t* topk_ids_host, const float* topk_weights_host, int T, int variant,
                          void* out_host, void* stream) {

@@ -111,6 +111,9 @@ struct Workspace {
 cudaError_t launch_route(const Workspace& ws, const int32_t* topk_ids, const float* topk_weights, int T, int k, int E,
                          const SelectorArgs& sel, int32_t* hist_out, double* eff_out, bool stats_only,
                          cudaStream_t stream);
+// router.cu
+cudaError_t launch_router_topk(const float* logits, int T, int E, int k, int32_t* ids, float* weights,
+                               cudaStream_t stream);
 // misc.cu
 cudaError_t launch_gather(const Workspace& ws, const __nv_bfloat16* x, int T, int k, int H, cudaStream_t stream);
 cudaError_t launch_reduce(const Workspace& ws, __nv_bfloat16* out, int T, int k, int H, cudaStream_t stream);

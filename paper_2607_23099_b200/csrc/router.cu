@@ -1,0 +1,102 @@
+// Router top-k: the step upstream of the expert layer.  The paper's end-to-end MoE-layer metric
+// (Section V) covers "router selection, routing-metadata construction, dispatch and fused-MoE
+// execution"; this kernel is the router selection.  Per token it picks the k largest of E router
+// logits (ties: the lower expert index) and turns the selected logits into routing weights with a
+// softmax over those k values, the gating the build's configurations use.
+//
+// One warp per token.  A lane keeps logits lane, lane + 32, ... (at most 32 of them, E <= 1024) as
+// order-preserving 32-bit keys; each of the k rounds takes the lane-local maximum of what is left
+// and a warp-wide maximum over 64-bit (key, ~index) pairs, so the result does not depend on the
+// schedule.  NaN logits sort below every number.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace damoe {
+
+namespace {
+
+constexpr int kRouterWarps = 8;  // tokens per CTA
+
+// Monotone map float -> uint32: a < b  <=>  key(a) < key(b); NaN -> 0 (below -inf).
+__device__ __forceinline__ uint32_t ordered_key(float f) {
+  if (f != f) return 0u;
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_to_float(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+
+__global__ void __launch_bounds__(kRouterWarps * 32) router_topk_kernel(const float* __restrict__ logits, int T, int E,
+                                                                       int k, int32_t* __restrict__ ids,
+                                                                       float* __restrict__ weights) {
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * kRouterWarps + (threadIdx.x >> 5);
+  pdl_wait();
+  pdl_launch_dependents();
+  if (t >= T) return;
+  const float* row = logits + static_cast<size_t>(t) * E;
+  uint32_t key[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const int e = i * 32 + lane;
+    key[i] = (e < E) ? ordered_key(__ldg(row + e)) : 0u;
+  }
+  uint32_t taken = 0u;  // bit i: this lane's i-th logit has been selected
+#pragma unroll
+  for (int i = 0; i < 32; ++i)
+    if (i * 32 + lane >= E) taken |= 1u << i;  // slots past E never compete
+
+  float my_logit = 0.f;  // lane j ends up with the j-th selected logit
+  int my_id = -1;
+  for (int j = 0; j < k; ++j) {
+    // (key, ~index) packed so that the maximum is the largest logit and, among equals, the lowest index
+    unsigned long long best = 0ull;
+    int best_i = -1;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      if (!((taken >> i) & 1u)) {
+        const unsigned long long c =
+            (static_cast<unsigned long long>(key[i]) << 32) | static_cast<uint32_t>(~static_cast<uint32_t>(i * 32 + lane));
+        if (best_i < 0 || c > best) {
+          best = c;
+          best_i = i;
+        }
+      }
+    }
+    // a lane with nothing left offers 0, which loses against any real candidate (~index > 0 for index < 2^32 - 1)
+    unsigned long long m = (best_i >= 0) ? best : 0ull;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      const unsigned long long o = __shfl_xor_sync(0xffffffffu, m, d);
+      m = o > m ? o : m;
+    }
+    if (best_i >= 0 && best == m) taken |= 1u << best_i;  // exactly one lane owns the winner: indices are distinct
+    if (lane == j) {
+      my_id = static_cast<int>(~static_cast<uint32_t>(m & 0xFFFFFFFFull));
+      my_logit = key_to_float(static_cast<uint32_t>(m >> 32));
+    }
+  }
+  // softmax over the k selected logits; the first selected one is the largest
+  const float top = __shfl_sync(0xffffffffu, my_logit, 0);
+  float ex = (lane < k) ? expf(my_logit - top) : 0.f;
+  if (lane < k && my_logit != my_logit) ex = 0.f;  // a NaN was selected only because fewer than k numbers exist
+  float sum = ex;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
+  if (lane < k) {
+    ids[static_cast<size_t>(t) * k + lane] = my_id;
+    weights[static_cast<size_t>(t) * k + lane] = __fdiv_rn(ex, sum);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_router_topk(const float* logits, int T, int E, int k, int32_t* ids, float* weights,
+                               cudaStream_t stream) {
+  const int grid = (T + kRouterWarps - 1) / kRouterWarps;
+  return launch_k(router_topk_kernel, dim3(grid), dim3(kRouterWarps * 32), 0, stream, logits, T, E, k, ids, weights);
+}
+
+}  // namespace damoe
