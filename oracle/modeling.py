@@ -15,7 +15,17 @@ What the paper fixes
   * an exemplar is the per-expert token-count vector sorted in descending order
     and scaled to unit L2 norm; with several samples the centroid is used
                                                                   (Section IV-A)
+  * besides the Dirichlet family the paper compares an exponential and a Beta family
+    of synthetic distributions, each parameterised to match a target eff_exp: the
+    exponential one by binary search, the Beta one by a brute-force search over its two
+    parameters on a grid of spacing 0.1; families are compared by cosine similarity of
+    the sorted, L2-normalised vectors                              (Section V, Fig. 14)
 Readings taken where the paper is silent
+  * the exponential family is p_i proportional to exp(-lambda * i), i = 0..E-1;
+  * the Beta family is p_i proportional to x_i with x_i drawn independently from
+    Beta(a, b) by a caller-supplied sampler; its search averages eff_exp over S draws per
+    grid point and takes the grid point closest to the target (first in row-major order
+    on ties);
   * Algorithm 1 applies eff_exp to the sampled probability vectors, as printed;
   * the Dirichlet draws come from a caller-supplied sampler, so the search can
     run on common random numbers and be deterministic;
@@ -85,3 +95,47 @@ def cosine(a, b) -> float:
     a = np.asarray(a, dtype=np.float64)
     b = np.asarray(b, dtype=np.float64)
     return float(np.dot(a, b) / (np.sqrt(np.dot(a, a)) * np.sqrt(np.dot(b, b))))
+
+
+def exponential_p(lam: float, E: int) -> np.ndarray:
+    """Exponential family: p_i proportional to exp(-lam * i), i = 0..E-1."""
+    z = -float(lam) * np.arange(E, dtype=np.float64)
+    w = np.exp(z - z.max())
+    return w / w.sum()
+
+
+def binary_search_exponential(target: float, E: int, iters: int = 80, lam_min: float = 0.0,
+                              lam_max: float = 64.0) -> float:
+    """Decay rate whose exponential distribution has eff_exp = target (eff_exp falls as lam grows)."""
+    lo, hi = lam_min, lam_max
+    mid = (lo + hi) / 2.0
+    for _ in range(iters):
+        mid = (lo + hi) / 2.0
+        if eff_exp(exponential_p(mid, E)) > target:
+            lo = mid          # too uniform: decay faster
+        else:
+            hi = mid
+    return mid
+
+
+def beta_p(a: float, b: float, E: int, S: int, draw) -> np.ndarray:
+    """Beta family: S probability vectors [S, E], p_i proportional to x_i ~ Beta(a, b).
+    ``draw(a, b, S, E)`` returns the raw Beta samples [S, E]."""
+    x = np.asarray(draw(a, b, S, E), dtype=np.float64)
+    return x / x.sum(axis=1, keepdims=True)
+
+
+def grid_search_beta(target: float, E: int, S: int, draw, step: float = 0.1, upper: float = 4.0):
+    """Brute-force search of (a, b) on the grid {step, 2 step, ..., upper}^2 for the Beta family
+    whose mean eff_exp over S draws is closest to the target."""
+    n = int(round(upper / step))
+    best = None
+    for ia in range(1, n + 1):
+        for ib in range(1, n + 1):
+            a, b = ia * step, ib * step
+            p = beta_p(a, b, E, S, draw)
+            v = sum(eff_exp(p[s]) for s in range(S)) / S
+            err = abs(v - target)
+            if best is None or err < best[0]:
+                best = (err, a, b)
+    return best[1], best[2]

@@ -83,3 +83,79 @@ def test_exemplar_is_sorted_unit_and_label_free():
     one = modeling.exemplar([[3, 0, 4]])
     np.testing.assert_allclose(one, [0.8, 0.6, 0.0])
     assert modeling.exemplar_q30([[3, 0, 4]]).tolist() == [round(0.8 * 2 ** 30), round(0.6 * 2 ** 30), 0]
+
+
+# ---- exponential and Beta families (paper Section V, the comparison of synthetic families) ----
+
+def _geometric_eff(lam, E):
+    # closed form of (sum r^i)^2 / sum r^(2i), r = exp(-lam)
+    r = np.exp(-lam)
+    if r == 1.0:
+        return float(E)
+    return ((1 - r ** E) / (1 - r)) ** 2 * (1 - r * r) / (1 - r ** (2 * E))
+
+
+def test_exponential_family_closed_form_and_limits():
+    for E in (8, 256):
+        for lam in (0.0, 1e-3, 0.05, 0.7, 5.0):
+            p = modeling.exponential_p(lam, E)
+            assert abs(p.sum() - 1.0) < 1e-12 and np.all(np.diff(p) <= 0)
+            assert np.isclose(modeling.eff_exp(p), _geometric_eff(lam, E), rtol=1e-10)
+    assert np.isclose(modeling.eff_exp(modeling.exponential_p(0.0, 64)), 64.0)
+    assert np.isclose(modeling.eff_exp(modeling.exponential_p(60.0, 64)), 1.0, rtol=1e-9)
+
+
+def test_exponential_bisection_reaches_the_target_and_is_monotone():
+    E = 256
+    lams = []
+    for X in (1.1, 1.5, 2.0, 4.0, 16.0):
+        target = modeling.ddist_target(E, X)
+        lam = modeling.binary_search_exponential(target, E)
+        assert np.isclose(_geometric_eff(lam, E), target, rtol=1e-9)
+        lams.append(lam)
+    assert all(a < b for a, b in zip(lams, lams[1:]))   # a more skewed target needs a faster decay
+    # large E, moderate decay: eff -> (1 + r) / (1 - r), i.e. lam = log((eff + 1) / (eff - 1))
+    assert np.isclose(modeling.binary_search_exponential(20.0, 4096), np.log(21.0 / 19.0), rtol=1e-6)
+
+
+def _beta_draw(seed):
+    def draw(a, b, S, E):
+        return np.random.default_rng(seed).beta(a, b, size=(S, E))
+    return draw
+
+
+def test_beta_family_law_of_large_numbers_and_grid_search():
+    # iid x_i: eff_exp / E -> E[x]^2 / E[x^2] = a (a + b + 1) / ((a + 1) (a + b))
+    E = 8192
+    for a, b in ((0.5, 0.5), (2.0, 3.0), (0.2, 1.5)):
+        p = modeling.beta_p(a, b, E, 4, _beta_draw(3))
+        assert np.allclose(p.sum(axis=1), 1.0)
+        got = np.mean([modeling.eff_exp(q) for q in p]) / E
+        assert np.isclose(got, a * (a + b + 1) / ((a + 1) * (a + b)), rtol=0.03)
+    # the brute-force search returns a grid point, and no other grid point is closer to the target
+    E, S, target = 64, 8, 24.0
+    a, b = modeling.grid_search_beta(target, E, S, _beta_draw(5), step=0.5, upper=2.0)
+    assert a in (0.5, 1.0, 1.5, 2.0) and b in (0.5, 1.0, 1.5, 2.0)
+
+    def mean_eff(a, b):
+        p = modeling.beta_p(a, b, E, S, _beta_draw(5))
+        return np.mean([modeling.eff_exp(q) for q in p])
+    best = abs(mean_eff(a, b) - target)
+    for aa in (0.5, 1.0, 1.5, 2.0):
+        for bb in (0.5, 1.0, 1.5, 2.0):
+            assert best <= abs(mean_eff(aa, bb) - target) + 1e-12
+
+
+def test_families_matched_to_one_target_have_similar_sorted_shapes():
+    # the paper compares the families by cosine similarity of sorted, L2-normalised vectors once they
+    # are matched to the same eff_exp; matched vectors must be close to each other, far from uniform
+    E, target = 256, 64.0
+    lam = modeling.binary_search_exponential(target, E)
+    pe = modeling.exponential_p(lam, E)
+    rng = np.random.default_rng(0)
+    alpha = (target - 1) / (E - target)           # closed-form Dirichlet inverse
+    pd = rng.dirichlet(np.full(E, alpha))
+    c = modeling.cosine(modeling.sorted_unit_vector(pe), modeling.sorted_unit_vector(pd))
+    u = modeling.cosine(modeling.sorted_unit_vector(pe), modeling.sorted_unit_vector(np.ones(E)))
+    assert c > 0.9 and c > u
+    assert np.isclose(u, np.sqrt(target / E), rtol=1e-6)   # cosine to uniform = sqrt(eff_exp / E)
