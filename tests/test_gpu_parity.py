@@ -403,6 +403,35 @@ def test_config3_kimi_shape_sampled_tokens(d):
     _sampled_full_size(d, 384, 8, 7168, 2048, 4096, [(1, 1.0, 21), (333, 0.3, 22), (4096, 5.0, 23)])
 
 
+def test_back_to_back_full_size_auto(d):
+    # The same overlap check on the DeepSeek-V3 shape through the shipped table: batch sizes that
+    # alternate between the fixed-variant launch, the plain branching kernel and the cluster-launched
+    # one, queued without synchronisation, must reproduce the results of the calls run alone.
+    E, k, H, I = 256, 8, 7168, 2048
+    W = di.MoEWeights(12345, E, H, I)
+    w13, w2 = W.materialize("cuda")
+    m = d.DAMoE(4096, k, E, H, I)
+    m.load_tuning_table(_table_bytes(E, k, H, I))
+    specs = [(64, 1.0), (1, 1.0), (4096, 0.05), (16, 10.0), (1024, 0.2), (8, 0.05), (256, 0.05), (2048, 1.0), (2, 1.0)]
+    ins, outs = [], []
+    for s_, (T, a) in enumerate(specs):
+        ids, w, _ = di.routing_batch(500 + s_, T, k, E, a)
+        ins.append((di.activations(500 + s_, T, H, "cuda"), torch.from_numpy(ids).cuda(), torch.from_numpy(w).cuda()))
+        outs.append(torch.empty(T, H, dtype=torch.bfloat16, device="cuda"))
+    torch.cuda.synchronize()
+    for rep in range(2):
+        for (x, ids, w), o in zip(ins, outs):
+            m.fused_moe(x, w13, w2, ids, w, d.VARIANT_AUTO, out=o)
+    torch.cuda.synchronize()
+    assert m.debug_fetch(specs[-1][0])["status"] == 0
+    for (T, a), (x, ids, w), o in zip(specs, ins, outs):
+        torch.cuda.synchronize()
+        alone = m.fused_moe(x, w13, w2, ids, w, d.VARIANT_AUTO)
+        torch.cuda.synchronize()
+        assert torch.equal(alone.view(torch.int16), o.view(torch.int16)), f"T={T}, alpha={a} differs when overlapped"
+    m.close()
+
+
 def test_dispatch_microbench_runs(d):
     r = d.dispatch_microbench(50)
     assert all(0 < v < 1e4 for v in r.values())
