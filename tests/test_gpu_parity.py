@@ -294,6 +294,43 @@ def test_capture_in_a_cuda_graph(d):
     m.close()
 
 
+@pytest.mark.parametrize("E,k,H,I,T,alpha", [(16, 4, 2048, 768, 300, 0.3), (8, 2, 4096, 1792, 130, 1.0),
+                                             (8, 2, 1152, 640, 97, 0.2), (32, 8, 1024, 256, 513, 0.1)])
+def test_other_shapes_every_available_variant(d, E, k, H, I, T, alpha):
+    # Shapes other than the paper's two models: K extents that are odd multiples of the K tile,
+    # odd numbers of 128-row weight tiles (the CTA-pair variants are then not offered), more slots
+    # per token than experts' tiles.  Sampled tokens against the oracle, every variant the context offers.
+    case = Case(31, T, E, k, H, I, alpha)
+    dev = "cuda:0"
+    w13, w2 = case.weights.materialize(dev)
+    m = d.DAMoE(T, k, E, H, I)
+    x, ids, w = case.x(dev), torch.from_numpy(case.ids).to(dev), torch.from_numpy(case.w).to(dev)
+    tokens = sorted(int(v) for v in np.random.default_rng(E).choice(T, size=3, replace=False))
+    ref_bits, _ = layer.moe_layer_bf16(bits16(case.x()), case.w13_bits, case.w2_bits, case.ids, case.w, E, tokens=tokens)
+    ref = codecs.bf16_decode(ref_bits)
+    pairs_possible = (H // 128) % 2 == 0 and (I // 128) % 2 == 0
+    ran = 0
+    first = None
+    for v in list(range(d.variant_count())) + [d.VARIANT_AUTO]:
+        info = d.variant_info(v) if v >= 0 else None
+        if info is not None and info["cta_group"] == 2 and not pairs_possible:
+            with pytest.raises(d.DamoeError):
+                m.fused_moe(x, w13, w2, ids, w, v)
+            continue
+        out = m.fused_moe(x, w13, w2, ids, w, v)
+        assert m.debug_fetch(T)["status"] == 0
+        got = codecs.bf16_decode(bits16(out))[np.asarray(tokens)]
+        assert rel_frobenius(got, ref) <= FROB_TOL, f"variant {v}"
+        assert max_scaled_err(got, ref) <= ELEM_TOL, f"variant {v}"
+        if first is None:
+            first = out.clone()
+        else:  # every variant accumulates an output element in the same K order: identical bits
+            assert torch.equal(first.view(torch.int16), out.view(torch.int16)), f"variant {v}"
+        ran += 1
+    assert ran >= 6
+    m.close()
+
+
 def test_back_to_back_calls_with_changing_routing(d):
     # The kernels of consecutive calls overlap through programmatic dependent launch, and a GEMM
     # reads the routing metadata and requests weight tiles before the kernel ahead of it has
