@@ -318,9 +318,16 @@ def compare_dispatch(m, d, cells, run, pk, reps=3):
         return a.elapsed_time(b) * 1e3
 
     rows = []
+    time.sleep(0.5)  # the timed loops before this comparison may have left the GPU power-capped
     for c in cells:
-        # warm every path once, then interleave the repetitions so that clock and cache drift
-        # hit AUTO, STATIC and the fixed variants alike
+        # let the GPU settle into this batch's own clock / power state (the batch before may have
+        # been a power-capped prefill-sized one), warm every path once, then interleave the
+        # repetitions so that clock and cache drift hit AUTO, STATIC and the fixed variants alike
+        t_settle, n_settle = time.perf_counter(), 0
+        while n_settle < 2 or time.perf_counter() - t_settle < 0.03:
+            run(c, d.VARIANT_AUTO)
+            torch.cuda.synchronize()
+            n_settle += 1
         run(c, d.VARIANT_AUTO)
         chosen = m.debug_fetch(c["T"])["variant_id"]
         run(c, d.VARIANT_STATIC)
