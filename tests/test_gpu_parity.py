@@ -133,6 +133,39 @@ def test_route_metadata_many_pairs(d):
     m.close()
 
 
+@pytest.mark.parametrize("E,k,T", [(1, 1, 5), (3, 2, 700), (77, 5, 41), (1000, 32, 64), (1024, 8, 2100), (33, 1, 1024)])
+def test_route_metadata_odd_and_maximal_expert_counts(d, E, k, T):
+    # Expert counts that are not multiples of a warp, the maximum the library takes (1024), one
+    # expert, k = 1 and k = 32: all integer outputs in full against the oracle, through both the
+    # single-kernel routing path (at most 1024 pairs) and the three-kernel one.
+    rng = np.random.default_rng(E * 131 + k)
+    ids = np.stack([rng.choice(E, size=k, replace=False) for _ in range(T)]).astype(np.int32)
+    if T > 8:                       # a few invalid ids: skipped, counted in the status word
+        ids[3, 0] = E
+        ids[7, k - 1] = -2
+    w = rng.random((T, k), dtype=np.float32)
+    H = I = 128
+    W = di.MoEWeights(9, E, H, I)
+    w13, w2 = W.materialize("cuda")
+    m = d.DAMoE(T, k, E, H, I)
+    x = di.activations(1, T, H, "cuda")
+    m.fused_moe(x, w13, w2, torch.from_numpy(ids).cuda(), torch.from_numpy(w).cuda(), d.VARIANT_AUTO)
+    meta = m.debug_fetch(T)
+    assert meta["status"] == (d.STATUS_BAD_ID if T > 8 else 0)
+    hist = route.histogram(ids, E)
+    off, perm, inv = route.offsets_and_permutation(ids, E)
+    nv = int(off[-1])
+    assert np.array_equal(meta["offsets"], off.astype(np.int32))
+    assert np.array_equal(meta["perm"][:nv], perm.astype(np.int32))
+    assert np.all(meta["perm"][nv:T * k] == -1)
+    assert np.array_equal(meta["inv"], inv.astype(np.int32))
+    assert np.array_equal(meta["tiles"], route.tile_counts(hist, d.tile_ns()).astype(np.int32))
+    h2, eff = m.route_stats(torch.from_numpy(ids).cuda())
+    assert np.array_equal(h2.cpu().numpy(), hist.astype(np.int32))
+    assert eff.item() == route.effective_experts(hist)[2]
+    m.close()
+
+
 def test_edge_cases(d):
     case = config0(seed=3, T=5)
     t = _device_case(case)
