@@ -524,6 +524,34 @@ def run_ours(args):
         from_logits_ms = l0.elapsed_time(l1)
         barrier()
 
+    # ---- prefill-sized workload only: the clock a library bf16 GEMM settles at under the same power cap ----
+    power_reference = None
+    if args.workload == "large_T" and rank == 0:
+        n = 8192
+        ga = torch.randn(n, n, device=device, dtype=torch.bfloat16)
+        gb = torch.randn(n, n, device=device, dtype=torch.bfloat16)
+        for _ in range(5):
+            torch.matmul(ga, gb)
+        torch.cuda.synchronize()
+        ref_sampler = ClockSampler(local)
+        time.sleep(0.25)
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        tr0 = time.perf_counter()
+        r0.record(stream)
+        n_mm = 0
+        while time.perf_counter() - tr0 < 3.0:
+            for _ in range(20):
+                torch.matmul(ga, gb)
+            n_mm += 20
+            torch.cuda.synchronize()
+        r1.record(stream)
+        torch.cuda.synchronize()
+        tr1 = time.perf_counter()
+        power_reference = dict(what="torch.matmul bf16 8192^3 looped for 3 s right after the layer loop (library GEMM: a reference for the clock under the power cap, not part of the path)",
+                               tflops=round(2.0 * n ** 3 * n_mm / (r0.elapsed_time(r1) * 1e-3) / 1e12, 1),
+                               clocks=ref_sampler.stop(tr0, tr1))
+        del ga, gb
+
     ms_total, e2e_ms, from_logits_ms = max_over_ranks([ms_total, e2e_ms, from_logits_ms], world, device)
     us_per_layer = ms_total * 1e3 / steps
     e2e_us = e2e_ms * 1e3 / steps
@@ -613,7 +641,7 @@ def run_ours(args):
                 from_logits=(dict(value=round(from_logits_ms * 1e3 / steps, 2), unit="us",
                                   what="router top-k + softmax over the selected logits, then the layer (logits [T,E] fp32 resident on the device)")
                              if from_logits_ms > 0 else None),
-                clocks=clocks, roofline=roofline, cpu_baseline=cpu, dispatch=dispatch,
+                clocks=clocks, power_reference=power_reference, roofline=roofline, cpu_baseline=cpu, dispatch=dispatch,
                 dispatch_overhead=overhead, device_status=status)
     print(json.dumps(line))
 
