@@ -85,8 +85,8 @@ enum { DAMOE_MODE_EXEMPLAR = 0, DAMOE_MODE_EFFEXP_BINS = 1, DAMOE_MODE_COST = 2 
  * code * scale.  The intermediate h is rounded to bf16 and re-quantised on the device to E4M3
  * with one scale per (pair, 128 channels): s = amax / 448 (1 when amax = 0), code =
  * e4m3_rn_sat(h / s), both in fp32.  `out` is bf16.  FP8 contexts offer variants 0..3
- * (N_v <= 128); a larger variant id is DAMOE_ERR_INVALID_ARG, and damoe_fused_moe_host is
- * bf16 only.
+ * (N_v <= 128); a larger variant id is DAMOE_ERR_INVALID_ARG; the host-buffer form for these
+ * contexts is damoe_fused_moe_host_fp8.
  */
 int damoe_create(damoe_ctx** ctx, int device, int max_T, int k, int E, int H, int I, int dtype);
 int damoe_destroy(damoe_ctx* ctx);
@@ -192,6 +192,15 @@ int damoe_debug_fetch_routing(damoe_ctx* ctx, int T, int32_t* topk_ids_host, flo
 int damoe_fused_moe_host(damoe_ctx* ctx, const void* x_host, const void* w13, const void* w2,
                          const int32_t* topk_ids_host, const float* topk_weights_host, int T,
                          int variant, void* out_host, void* stream);
+
+/*
+ * The same for FP8 contexts: xq_host [T,H] one-byte E4M3 codes and x_scale_host [T, H/128]
+ * float32 group scales on the host; the weight scales are those of the last
+ * damoe_set_fp8_scales call (its activation-scale pointer is not used by this call).
+ */
+int damoe_fused_moe_host_fp8(damoe_ctx* ctx, const void* xq_host, const float* x_scale_host, const void* w13,
+                             const void* w2, const int32_t* topk_ids_host, const float* topk_weights_host, int T,
+                             int variant, void* out_host, void* stream);
 
 /* FP8 block scales (dtype == DAMOE_FP8_E4M3_BLOCK128 only): x_scale dev [T, H/128],
  * w13_scale dev [E, 2I/128, H/128], w2_scale dev [E, H/128, I/128], all float32, row-major.

@@ -27,7 +27,7 @@ EXPORTS = [
     "damoe_fused_moe_host", "damoe_set_fp8_scales", "damoe_load_tuning_table", "damoe_set_dispatch",
     "damoe_variant_count", "damoe_variant_info", "damoe_debug_fetch", "damoe_dispatch_microbench",
     "damoe_set_profiling", "damoe_get_stage_ms", "damoe_route_stats_noalloc", "damoe_set_selector_mode",
-    "damoe_router_topk", "damoe_moe_from_logits", "damoe_debug_fetch_routing",
+    "damoe_router_topk", "damoe_moe_from_logits", "damoe_debug_fetch_routing", "damoe_fused_moe_host_fp8",
 ]
 
 
@@ -45,6 +45,7 @@ def _load() -> ctypes.CDLL:
     lib.damoe_route_stats.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     lib.damoe_fused_moe.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
     lib.damoe_fused_moe_host.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
+    lib.damoe_fused_moe_host_fp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
     lib.damoe_router_topk.argtypes = [vp, vp, i32, vp, vp, vp]
     lib.damoe_moe_from_logits.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, vp]
     lib.damoe_debug_fetch_routing.argtypes = [vp, i32, vp, vp]
@@ -196,6 +197,16 @@ class DAMoE:
         self._check(_lib.damoe_fused_moe_host(self._ctx, _ptr(x_host), _ptr(w13), _ptr(w2), _ptr(topk_ids_host),
                                               _ptr(topk_weights_host), T, variant, _ptr(out_host),
                                               _stream_ptr(stream)))
+        return out_host
+
+    def fused_moe_host_fp8(self, xq_host, x_scale_host, w13, w2, topk_ids_host, topk_weights_host,
+                           variant: int = VARIANT_AUTO, out_host=None, stream=None):
+        T = xq_host.shape[0]
+        if out_host is None:
+            out_host = torch.empty(T, self.H, dtype=torch.bfloat16).pin_memory()
+        self._check(_lib.damoe_fused_moe_host_fp8(self._ctx, _ptr(xq_host), _ptr(x_scale_host), _ptr(w13), _ptr(w2),
+                                                  _ptr(topk_ids_host), _ptr(topk_weights_host), T, variant,
+                                                  _ptr(out_host), _stream_ptr(stream)))
         return out_host
 
     def set_fp8_scales(self, x_scale, w13_scale, w2_scale):

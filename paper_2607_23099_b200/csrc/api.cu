@@ -720,7 +720,7 @@ int damoe_fused_moe_host(damoe_ctx* c, const void* x_host, const void* w13, cons
   if (T == 0) return DAMOE_OK;
   if (T < 0 || T > c->max_T) return fail(c, DAMOE_ERR_INVALID_ARG, "T=%d outside [0, %d]", T, c->max_T);
   if (!x_host || !topk_ids_host || !topk_weights_host || !out_host) return fail(c, DAMOE_ERR_INVALID_ARG, "null pointer");
-  if (c->dtype != DAMOE_BF16) return fail(c, DAMOE_ERR_UNSUPPORTED_SHAPE, "host-buffer entry point is bf16 only");
+  if (c->dtype != DAMOE_BF16) return fail(c, DAMOE_ERR_UNSUPPORTED_SHAPE, "FP8 contexts use damoe_fused_moe_host_fp8");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   DAMOE_CUDA(c, cudaSetDevice(c->device));
   const size_t P = static_cast<size_t>(T) * c->k;
@@ -729,6 +729,37 @@ int damoe_fused_moe_host(damoe_ctx* c, const void* x_host, const void* w13, cons
   DAMOE_CUDA(c, cudaMemcpyAsync(c->st_w, topk_weights_host, 4 * P, cudaMemcpyHostToDevice, st));
   int rc = damoe_fused_moe(c, c->st_x, w13, w2, static_cast<const int32_t*>(c->st_ids),
                            static_cast<const float*>(c->st_w), T, variant, c->st_out, stream);
+  if (rc != DAMOE_OK) return rc;
+  DAMOE_CUDA(c, cudaMemcpyAsync(out_host, c->st_out, 2 * static_cast<size_t>(T) * c->H, cudaMemcpyDeviceToHost, st));
+  DAMOE_CUDA(c, cudaStreamSynchronize(st));
+  return DAMOE_OK;
+}
+
+int damoe_fused_moe_host_fp8(damoe_ctx* c, const void* xq_host, const float* x_scale_host, const void* w13, const void* w2,
+                             const int32_t* topk_ids_host, const float* topk_weights_host, int T, int variant,
+                             void* out_host, void* stream) {
+  if (!c) return DAMOE_ERR_INVALID_ARG;
+  if (T == 0) return DAMOE_OK;
+  if (T < 0 || T > c->max_T) return fail(c, DAMOE_ERR_INVALID_ARG, "T=%d outside [0, %d]", T, c->max_T);
+  if (!xq_host || !x_scale_host || !topk_ids_host || !topk_weights_host || !out_host)
+    return fail(c, DAMOE_ERR_INVALID_ARG, "null pointer");
+  if (c->dtype != DAMOE_FP8_E4M3_BLOCK128) return fail(c, DAMOE_ERR_INVALID_ARG, "context is not FP8");
+  if (!c->w13_scale || !c->w2_scale) return fail(c, DAMOE_ERR_INVALID_ARG, "weight scales not set (damoe_set_fp8_scales)");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DAMOE_CUDA(c, cudaSetDevice(c->device));
+  const size_t P = static_cast<size_t>(T) * c->k;
+  const size_t nx = static_cast<size_t>(T) * c->H;  // codes; the scales follow them in the staging buffer
+  uint8_t* sx = static_cast<uint8_t*>(c->st_x);
+  float* sxs = reinterpret_cast<float*>(sx + nx);
+  DAMOE_CUDA(c, cudaMemcpyAsync(sx, xq_host, nx, cudaMemcpyHostToDevice, st));
+  DAMOE_CUDA(c, cudaMemcpyAsync(sxs, x_scale_host, 4 * nx / 128, cudaMemcpyHostToDevice, st));
+  DAMOE_CUDA(c, cudaMemcpyAsync(c->st_ids, topk_ids_host, 4 * P, cudaMemcpyHostToDevice, st));
+  DAMOE_CUDA(c, cudaMemcpyAsync(c->st_w, topk_weights_host, 4 * P, cudaMemcpyHostToDevice, st));
+  const float* caller_scale = c->x_scale;
+  c->x_scale = sxs;
+  const int rc = damoe_fused_moe(c, sx, w13, w2, static_cast<const int32_t*>(c->st_ids),
+                                 static_cast<const float*>(c->st_w), T, variant, c->st_out, stream);
+  c->x_scale = caller_scale;
   if (rc != DAMOE_OK) return rc;
   DAMOE_CUDA(c, cudaMemcpyAsync(out_host, c->st_out, 2 * static_cast<size_t>(T) * c->H, cudaMemcpyDeviceToHost, st));
   DAMOE_CUDA(c, cudaStreamSynchronize(st));

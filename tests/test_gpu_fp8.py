@@ -115,3 +115,22 @@ def test_fp8_config4_shape_sampled_tokens(d):
         tokens = [int(v) for v in np.random.default_rng(seed).choice(T, size=2, replace=False)]
         _check(out, _oracle(case, wq, tokens=tokens), tokens=tokens)
     m.close()
+
+
+def test_fp8_host_buffer_entry_point(d):
+    E, k, H, I, T = 8, 2, 1024, 512, 64
+    case = Fp8Case(9, T, E, k, H, I, 1.0)
+    wq = case.W.materialize_fp8("cuda:0")
+    w13q, w13s, w2q, w2s = wq
+    m = d.DAMoE(T, k, E, H, I, dtype=d.FP8_E4M3_BLOCK128)
+    out_dev, _ = _run(d, m, case, wq, d.VARIANT_AUTO)
+    # the same call with the per-step tensors on the host; the activation-scale pointer given to
+    # set_fp8_scales is not used by it
+    dummy = torch.zeros_like(case.xs)
+    m._check(d._lib.damoe_set_fp8_scales(m._ctx, d._ptr(dummy), d._ptr(w13s), d._ptr(w2s)))
+    out_host = m.fused_moe_host_fp8(case.xq.cpu().pin_memory(), case.xs.cpu().pin_memory(), w13q, w2q,
+                                    torch.from_numpy(case.ids).pin_memory(), torch.from_numpy(case.w).pin_memory(),
+                                    d.VARIANT_AUTO)
+    assert torch.equal(out_host.view(torch.int16), out_dev.cpu().view(torch.int16))
+    _check(out_host, _oracle(case, wq))
+    m.close()
